@@ -319,7 +319,8 @@ int spo_path_scores(const float *logits, int64_t ld, const int32_t *targets,
  * Reading (Algorithm 3 prints argmin^K; the text says top-k, k = paths retained):
  *   keep the k LARGEST.
  * Reading (silent): ties -> lower path index first; NaN ranks below every number;
- *   k > N_b fills N_b entries and pads with -1; posterior treats NaN as -inf.
+ *   k > N_b fills N_b entries and pads with -1; posterior treats NaN as -inf, and is 0
+ *   everywhere when no score of the prompt is above -inf.
  * kept_idx: [B, k] global path ids in descending score; kept_post: [B, k] or NULL.
  * ---------------------------------------------------------------------------------- */
 static int score_before(const float *s, int a, int b) /* 1 if a ranks before b */
@@ -347,13 +348,14 @@ int spo_prune_topk(const float *scores, const int32_t *ppo, int n_prompts, int k
         }
         double m = -INFINITY, denom = 0.0;
         for (int i = 0; i < n; ++i) if (!isnan(scores[lo + i]) && scores[lo + i] > m) m = scores[lo + i];
-        for (int i = 0; i < n; ++i) if (!isnan(scores[lo + i])) denom += exp((double)scores[lo + i] - m);
+        if (m > -INFINITY)
+            for (int i = 0; i < n; ++i) if (!isnan(scores[lo + i])) denom += exp((double)scores[lo + i] - m);
         for (int j = 0; j < k; ++j) {
             if (j < n) {
                 kept_idx[b * k + j] = ord[j];
                 if (kept_post) {
                     const float sc = scores[ord[j]];
-                    kept_post[b * k + j] = isnan(sc) ? 0.0f : (float)(exp((double)sc - m) / denom);
+                    kept_post[b * k + j] = (isnan(sc) || !(denom > 0.0)) ? 0.0f : (float)(exp((double)sc - m) / denom);
                 }
             } else {
                 kept_idx[b * k + j] = -1;

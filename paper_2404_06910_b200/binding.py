@@ -1,0 +1,209 @@
+"""ctypes binding of libsp_b200.so (declared in include/sp.h).
+
+Argument marshalling only: every function forwards raw device pointers and sizes to the
+C ABI entry point of the same name.  torch is used for device memory and streams.
+There is no fallback: if the CUDA library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsp_b200.so")
+
+SP_OK = 0
+SP_ERR_INVALID_ARG, SP_ERR_UNSUPPORTED, SP_ERR_WORKSPACE, SP_ERR_CUDA, SP_ERR_TIMEOUT = 1, 2, 3, 4, 5
+SP_F32, SP_BF16 = 0, 1
+SP_ROWS_ALL, SP_ROWS_QUERY_ONLY = 0, 1
+SP_POS_EQUILIBRIUM, SP_POS_LEFT_ALIGNED = 0, 1
+SP_ROPE_HALF_SPLIT, SP_ROPE_INTERLEAVED = 0, 1
+
+EXPORTS = (
+    "sp_last_error", "sp_version", "sp_positions", "sp_rope_apply",
+    "sp_prefill_workspace_bytes", "sp_superpose_prefill",
+    "sp_path_scores_workspace_bytes", "sp_path_scores", "sp_prune_topk",
+    "sp_decode_workspace_bytes", "sp_pruned_decode", "sp_check_status",
+)
+
+
+class SpError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"sp status {code}: {message}")
+        self.code = code
+
+
+class _CLayout(ctypes.Structure):
+    _fields_ = [
+        ("n_prompts", ctypes.c_int32), ("n_paths", ctypes.c_int32),
+        ("prompt_path_off", ctypes.c_void_p), ("pre_start", ctypes.c_void_p),
+        ("pre_len", ctypes.c_void_p), ("path_start", ctypes.c_void_p),
+        ("doc_len", ctypes.c_void_p), ("qry_len", ctypes.c_void_p),
+        ("total_tokens", ctypes.c_int64),
+        ("max_pre_len", ctypes.c_int32), ("max_path_len", ctypes.c_int32),
+    ]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2404_06910_b200.build` "
+            "(there is no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    c_int, c_i64, c_f, c_d, vp, sz = (ctypes.c_int, ctypes.c_int64, ctypes.c_float, ctypes.c_double,
+                                      ctypes.c_void_p, ctypes.c_size_t)
+    lp = ctypes.POINTER(_CLayout)
+    lib.sp_last_error.restype = ctypes.c_char_p
+    lib.sp_version.restype = ctypes.c_char_p
+    lib.sp_positions.argtypes = [c_int, c_int, c_int, c_int, vp, c_int, vp, ctypes.POINTER(c_d), ctypes.POINTER(c_d)]
+    lib.sp_rope_apply.argtypes = [vp, vp, c_i64, c_i64, c_int, c_int, c_int, c_d, c_int, c_int, vp]
+    lib.sp_prefill_workspace_bytes.argtypes = [c_int] * 7
+    lib.sp_prefill_workspace_bytes.restype = sz
+    lib.sp_superpose_prefill.argtypes = [vp, vp, vp, lp, c_int, c_int, c_int, c_f, c_int, vp, vp, vp, sz, c_int, vp]
+    lib.sp_path_scores_workspace_bytes.argtypes = [c_i64]
+    lib.sp_path_scores_workspace_bytes.restype = sz
+    lib.sp_path_scores.argtypes = [vp, c_i64, vp, vp, c_i64, c_int, c_int, vp, vp, vp, vp, vp, sz, c_int, vp]
+    lib.sp_prune_topk.argtypes = [vp, vp, c_int, c_int, vp, vp, vp]
+    lib.sp_decode_workspace_bytes.argtypes = [c_int, c_int, c_int]
+    lib.sp_decode_workspace_bytes.restype = sz
+    lib.sp_pruned_decode.argtypes = [vp, vp, vp, lp, vp, c_int, vp, vp, vp, c_int, c_i64, c_int, c_int, c_int,
+                                     c_f, vp, vp, vp, sz, c_int, vp]
+    lib.sp_check_status.argtypes = [vp, vp]
+    for name in EXPORTS:
+        getattr(lib, name)          # raises AttributeError if a declared symbol is not exported
+    return lib
+
+
+lib = _load()
+
+
+def _check(rc: int):
+    if rc != SP_OK:
+        raise SpError(rc, lib.sp_last_error().decode())
+
+
+def dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return SP_F32
+    if t.dtype == torch.bfloat16:
+        return SP_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors must be contiguous"
+    return t.data_ptr()
+
+
+def _nbytes(t):
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+@dataclass
+class DeviceLayout:
+    """sp_layout with its index arrays resident on the device."""
+    c: _CLayout
+    arrays: tuple          # keeps the device tensors alive
+    n_prompts: int
+    n_paths: int
+    total_tokens: int
+    max_pre_len: int
+    max_path_len: int
+
+    @property
+    def prompt_path_off(self):
+        return self.arrays[0]
+
+    @staticmethod
+    def from_host(lay, device="cuda") -> "DeviceLayout":
+        def dev(a):
+            return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
+        arrs = tuple(dev(a) for a in (lay.prompt_path_off, lay.pre_start, lay.pre_len,
+                                      lay.path_start, lay.doc_len, lay.qry_len))
+        c = _CLayout(lay.n_prompts, lay.n_paths, *[a.data_ptr() for a in arrs],
+                     lay.total_tokens, lay.max_pre_len, lay.max_path_len)
+        return DeviceLayout(c, arrs, lay.n_prompts, lay.n_paths, lay.total_tokens,
+                            lay.max_pre_len, lay.max_path_len)
+
+
+def sp_version() -> str:
+    return lib.sp_version().decode()
+
+
+def sp_positions(pre_len: int, doc_lens, qry_len: int, scheme: int = SP_POS_EQUILIBRIUM, q_mode: int = 0):
+    """Host call.  Returns (pos float32 [P + sum(L) + N*Q], S, next_pos)."""
+    L = np.ascontiguousarray(doc_lens, dtype=np.int32)
+    pos = np.empty(int(pre_len + L.sum() + len(L) * qry_len), dtype=np.float32)
+    S, nxt = ctypes.c_double(), ctypes.c_double()
+    _check(lib.sp_positions(scheme, q_mode, pre_len, len(L), L.ctypes.data, qry_len, pos.ctypes.data,
+                            ctypes.byref(S), ctypes.byref(nxt)))
+    return pos, S.value, nxt.value
+
+
+def sp_rope_apply(x: torch.Tensor, pos: torch.Tensor, n_heads: int, head_dim: int, *, n_tokens=None,
+                  ld_token=None, rot_dim=None, base: float = 10000.0, pairing: int = SP_ROPE_HALF_SPLIT,
+                  stream=None):
+    """In place on x ([n_tokens, n_heads, head_dim] with token stride ld_token elements)."""
+    n = pos.numel() if n_tokens is None else n_tokens
+    ld = n_heads * head_dim if ld_token is None else ld_token
+    _check(lib.sp_rope_apply(x.data_ptr(), pos.data_ptr(), n, ld, n_heads, head_dim,
+                             head_dim if rot_dim is None else rot_dim, base, pairing, dtype_code(x),
+                             _stream(stream)))
+
+
+def sp_prefill_workspace_bytes(lay: DeviceLayout, n_heads: int, head_dim: int, dtype: int) -> int:
+    return int(lib.sp_prefill_workspace_bytes(lay.n_prompts, lay.n_paths, lay.max_pre_len, lay.max_path_len,
+                                              n_heads, head_dim, dtype))
+
+
+def sp_superpose_prefill(q, k, v, lay: DeviceLayout, scale: float, out, lse=None, ws=None,
+                         rows: int = SP_ROWS_ALL, stream=None):
+    T, H, D = q.shape
+    Hkv = k.shape[1]
+    _check(lib.sp_superpose_prefill(_ptr(q), _ptr(k), _ptr(v), ctypes.byref(lay.c), H, Hkv, D, scale, rows,
+                                    _ptr(out), _ptr(lse), _ptr(ws), _nbytes(ws), dtype_code(q), _stream(stream)))
+
+
+def sp_path_scores_workspace_bytes(n_rows: int) -> int:
+    return int(lib.sp_path_scores_workspace_bytes(n_rows))
+
+
+def sp_path_scores(logits, targets, row_off, scores, prior=None, weight=None, row_logp=None, ws=None,
+                   stream=None):
+    R, V = logits.shape
+    _check(lib.sp_path_scores(logits.data_ptr(), logits.stride(0) if R else V, _ptr(targets), _ptr(row_off), R,
+                              row_off.numel() - 1, V, _ptr(prior), _ptr(weight), _ptr(scores), _ptr(row_logp),
+                              _ptr(ws), _nbytes(ws), dtype_code(logits), _stream(stream)))
+
+
+def sp_prune_topk(scores, prompt_path_off, k: int, kept_idx, kept_post=None, stream=None):
+    _check(lib.sp_prune_topk(_ptr(scores), _ptr(prompt_path_off), prompt_path_off.numel() - 1, k,
+                             _ptr(kept_idx), _ptr(kept_post), _stream(stream)))
+
+
+def sp_decode_workspace_bytes(n_prompts: int, n_heads: int, head_dim: int) -> int:
+    return int(lib.sp_decode_workspace_bytes(n_prompts, n_heads, head_dim))
+
+
+def sp_pruned_decode(q, k_cache, v_cache, lay: DeviceLayout, kept_idx, k: int, tail_k, tail_v, tail_len,
+                     tail_cap: int, scale: float, out, lse=None, ws=None, max_keys: int = 0, stream=None):
+    B, H, D = q.shape
+    Hkv = k_cache.shape[1]
+    _check(lib.sp_pruned_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), ctypes.byref(lay.c), _ptr(kept_idx), k,
+                                _ptr(tail_k), _ptr(tail_v), _ptr(tail_len), tail_cap, max_keys, H, Hkv, D, scale,
+                                _ptr(out), _ptr(lse), _ptr(ws), _nbytes(ws), dtype_code(q), _stream(stream)))
+
+
+def sp_check_status(ws, stream=None) -> None:
+    _check(lib.sp_check_status(_ptr(ws), _stream(stream)))

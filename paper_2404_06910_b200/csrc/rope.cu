@@ -1,0 +1,170 @@
+// sp_rope_apply: rotary position encoding at real-valued positions (Section 3.2.2,
+// footnote on RoPE: the sinusoid's argument is evaluated at the interpolated position).
+//
+// HBM-bound: one read and one write of x.  The rot_dim/2 angles of a token are the same
+// for all of its heads, so each (token, pair) angle is evaluated once, in fp64, by one
+// thread and shared through shared memory; the data pass is 16-byte vector loads/stores.
+#include "common.cuh"
+
+namespace sp {
+
+struct RopeFreq {
+    double inv_freq[128];   // base^(-2m/rot_dim), m < rot_dim/2 <= 128, computed on the host
+};
+
+constexpr int kRopeThreads = 256;
+constexpr int kRopeTokens = 4;   // tokens per block iteration
+
+template <typename T> struct Pack;
+template <> struct Pack<__nv_bfloat16> {
+    static constexpr int N = 8;
+    __device__ static void load(const __nv_bfloat16 *p, float (&f)[8]) { Vec<__nv_bfloat16>::load(p, f); }
+    __device__ static void store(__nv_bfloat16 *p, const float (&f)[8]) {
+        uint4 w;
+        w.x = pack_bf16x2(f[0], f[1]); w.y = pack_bf16x2(f[2], f[3]);
+        w.z = pack_bf16x2(f[4], f[5]); w.w = pack_bf16x2(f[6], f[7]);
+        *reinterpret_cast<uint4 *>(p) = w;
+    }
+};
+template <> struct Pack<float> {
+    static constexpr int N = 4;
+    __device__ static void load(const float *p, float (&f)[4]) { Vec<float>::load(p, f); }
+    __device__ static void store(float *p, const float (&f)[4]) {
+        *reinterpret_cast<float4 *>(p) = make_float4(f[0], f[1], f[2], f[3]);
+    }
+};
+
+// VEC: 16-byte accesses (requires alignment and divisibility, checked by the host).
+template <typename T, bool VEC>
+__global__ void __launch_bounds__(kRopeThreads)
+rope_kernel(T *__restrict__ x, const float *__restrict__ pos, int64_t n_tokens, int64_t ld_token,
+            int n_heads, int head_dim, int rot_dim, int pairing, const __grid_constant__ RopeFreq fr)
+{
+    __shared__ float2 cs[kRopeTokens][128];   // (cos, sin) per (token, pair)
+    const int half = rot_dim >> 1;
+    const int64_t n_groups = (n_tokens + kRopeTokens - 1) / kRopeTokens;
+
+    for (int64_t g = blockIdx.x; g < n_groups; g += gridDim.x) {
+        const int64_t t0 = g * kRopeTokens;
+        const int nt = (int)min((int64_t)kRopeTokens, n_tokens - t0);
+        __syncthreads();
+        for (int i = threadIdx.x; i < nt * half; i += kRopeThreads) {
+            const int t = i / half, m = i - t * half;
+            double s, c;
+            sincos((double)pos[t0 + t] * fr.inv_freq[m], &s, &c);
+            cs[t][m] = make_float2((float)c, (float)s);
+        }
+        __syncthreads();
+
+        if (VEC) {
+            constexpr int N = Pack<T>::N;
+            if (pairing == SP_ROPE_HALF_SPLIT) {
+                const int vec_per_head = half / N;
+                const int items = nt * n_heads * vec_per_head;
+                for (int i = threadIdx.x; i < items; i += kRopeThreads) {
+                    const int t = i / (n_heads * vec_per_head);
+                    const int r = i - t * (n_heads * vec_per_head);
+                    const int h = r / vec_per_head, m0 = (r - h * vec_per_head) * N;
+                    T *pa = x + (t0 + t) * ld_token + (int64_t)h * head_dim + m0;
+                    T *pb = pa + half;
+                    float a[N], b[N];
+                    Pack<T>::load(pa, a);
+                    Pack<T>::load(pb, b);
+#pragma unroll
+                    for (int j = 0; j < N; ++j) {
+                        const float2 w = cs[t][m0 + j];
+                        const float na = a[j] * w.x - b[j] * w.y;
+                        const float nb = a[j] * w.y + b[j] * w.x;
+                        a[j] = na; b[j] = nb;
+                    }
+                    Pack<T>::store(pa, a);
+                    Pack<T>::store(pb, b);
+                }
+            } else {
+                const int vec_per_head = rot_dim / N;
+                const int items = nt * n_heads * vec_per_head;
+                for (int i = threadIdx.x; i < items; i += kRopeThreads) {
+                    const int t = i / (n_heads * vec_per_head);
+                    const int r = i - t * (n_heads * vec_per_head);
+                    const int h = r / vec_per_head, e0 = (r - h * vec_per_head) * N;
+                    T *p = x + (t0 + t) * ld_token + (int64_t)h * head_dim + e0;
+                    float f[N];
+                    Pack<T>::load(p, f);
+#pragma unroll
+                    for (int j = 0; j < N; j += 2) {
+                        const float2 w = cs[t][(e0 + j) >> 1];
+                        const float na = f[j] * w.x - f[j + 1] * w.y;
+                        const float nb = f[j] * w.y + f[j + 1] * w.x;
+                        f[j] = na; f[j + 1] = nb;
+                    }
+                    Pack<T>::store(p, f);
+                }
+            }
+        } else {
+            const int items = nt * n_heads * half;
+            for (int i = threadIdx.x; i < items; i += kRopeThreads) {
+                const int t = i / (n_heads * half);
+                const int r = i - t * (n_heads * half);
+                const int h = r / half, m = r - h * half;
+                T *base = x + (t0 + t) * ld_token + (int64_t)h * head_dim;
+                T *pa = base + (pairing == SP_ROPE_HALF_SPLIT ? m : 2 * m);
+                T *pb = base + (pairing == SP_ROPE_HALF_SPLIT ? m + half : 2 * m + 1);
+                const float a = to_float(*pa), b = to_float(*pb);
+                const float2 w = cs[t][m];
+                store_val(pa, a * w.x - b * w.y);
+                store_val(pb, a * w.y + b * w.x);
+            }
+        }
+    }
+}
+
+template <typename T>
+static int launch_rope(void *x, const float *pos, int64_t n_tokens, int64_t ld_token, int n_heads,
+                       int head_dim, int rot_dim, int pairing, const RopeFreq &fr, cudaStream_t st)
+{
+    constexpr int N = Pack<T>::N;
+    const int half = rot_dim / 2;
+    const bool vec = aligned16(x) && (ld_token % N == 0) && (head_dim % N == 0) &&
+                     (pairing == SP_ROPE_HALF_SPLIT ? (half % N == 0) : (rot_dim % N == 0));
+    const int64_t n_groups = (n_tokens + kRopeTokens - 1) / kRopeTokens;
+    const int grid = (int)std::min<int64_t>(n_groups, (int64_t)kNumSMs * 16);
+    if (vec)
+        rope_kernel<T, true><<<grid, kRopeThreads, 0, st>>>((T *)x, pos, n_tokens, ld_token, n_heads,
+                                                            head_dim, rot_dim, pairing, fr);
+    else
+        rope_kernel<T, false><<<grid, kRopeThreads, 0, st>>>((T *)x, pos, n_tokens, ld_token, n_heads,
+                                                             head_dim, rot_dim, pairing, fr);
+    SP_CUDA(cudaGetLastError());
+    return SP_OK;
+}
+
+}  // namespace sp
+
+extern "C" int sp_rope_apply(void *x, const float *pos, int64_t n_tokens, int64_t ld_token,
+                             int n_heads, int head_dim, int rot_dim, double base, int pairing,
+                             int dtype, void *stream)
+{
+    using namespace sp;
+    SP_REQUIRE(dtype == SP_F32 || dtype == SP_BF16, SP_ERR_INVALID_ARG, "sp_rope_apply: unknown dtype %d", dtype);
+    SP_REQUIRE(n_tokens >= 0, SP_ERR_INVALID_ARG, "sp_rope_apply: n_tokens < 0");
+    SP_REQUIRE(n_heads > 0 && head_dim > 0 && head_dim <= 256, SP_ERR_INVALID_ARG,
+               "sp_rope_apply: n_heads %d / head_dim %d out of range", n_heads, head_dim);
+    SP_REQUIRE(rot_dim >= 2 && rot_dim <= head_dim && (rot_dim & 1) == 0, SP_ERR_INVALID_ARG,
+               "sp_rope_apply: rot_dim %d must be even and in [2, head_dim]", rot_dim);
+    SP_REQUIRE(pairing == SP_ROPE_HALF_SPLIT || pairing == SP_ROPE_INTERLEAVED, SP_ERR_INVALID_ARG,
+               "sp_rope_apply: unknown pairing %d", pairing);
+    SP_REQUIRE(ld_token >= (int64_t)n_heads * head_dim, SP_ERR_INVALID_ARG,
+               "sp_rope_apply: ld_token %lld < n_heads*head_dim", (long long)ld_token);
+    SP_REQUIRE(base > 0.0, SP_ERR_INVALID_ARG, "sp_rope_apply: base must be positive");
+    if (n_tokens == 0) return SP_OK;
+    SP_REQUIRE(x != nullptr && pos != nullptr, SP_ERR_INVALID_ARG, "sp_rope_apply: NULL pointer");
+    SP_REQUIRE((reinterpret_cast<uintptr_t>(x) % elt_bytes(dtype)) == 0, SP_ERR_INVALID_ARG,
+               "sp_rope_apply: x is not aligned to its element size");
+
+    RopeFreq fr;
+    for (int m = 0; m < rot_dim / 2; ++m) fr.inv_freq[m] = std::pow(base, -2.0 * m / rot_dim);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return dtype == SP_F32
+               ? launch_rope<float>(x, pos, n_tokens, ld_token, n_heads, head_dim, rot_dim, pairing, fr, st)
+               : launch_rope<__nv_bfloat16>(x, pos, n_tokens, ld_token, n_heads, head_dim, rot_dim, pairing, fr, st);
+}
