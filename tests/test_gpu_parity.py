@@ -1,0 +1,402 @@
+"""GPU parity: every entry point of the C ABI against the CPU oracle, element by element on
+the same seeded inputs, at sizes that span several tiles and ragged tails, plus edge cases.
+
+Tolerances (stated by the target): attention outputs rel-L2 <= 1e-2 for bf16 and <= 1e-5
+for fp32; |sum_t row_logp| within 1e-3 * query length; top-k indices bit-exact."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2404_06910_b200 as sp
+from helpers import dev, f32, positions_for, rel_l2, workspace
+from workloads import (CONFIGS, build_layout, draw_decode_inputs, draw_lengths, draw_logits,
+                       draw_prior_weight, draw_qkv, draw_targets)
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-5, "bf16": 1e-2}
+TDT = {"f32": torch.float32, "bf16": torch.bfloat16}
+
+
+def _rng(seed):
+    g = torch.Generator()
+    g.manual_seed(seed)
+    return g
+
+
+def _randn(shape, dtype, seed, std=1.0):
+    return (torch.randn(*shape, generator=_rng(seed)) * std).to(TDT[dtype])
+
+
+# ------------------------------------------------------------------------- RoPE
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("pairing", [0, 1])
+@pytest.mark.parametrize("H,D,rot", [(4, 64, 64), (32, 128, 128), (3, 128, 64), (2, 24, 12)])
+def test_rope_parity(dtype, pairing, H, D, rot):
+    n = 301
+    x = _randn((n, H, D), dtype, 7)
+    pos = (torch.rand(n, generator=_rng(8)) * 700).float()
+    ref = oracle.rope(f32(x), pos.numpy(), rot_dim=rot, pairing=pairing)
+    xd = dev(x)
+    sp.sp_rope_apply(xd, dev(pos), H, D, rot_dim=rot, pairing=pairing)
+    got = f32(xd)
+    if dtype == "f32":
+        np.testing.assert_allclose(got, ref, rtol=0, atol=4e-6)
+    else:   # one bf16 rounding of the fp32 result
+        assert np.all(np.abs(got - ref) <= np.abs(ref) * 2.0 ** -8 * 1.02 + 1e-6)
+
+
+def test_rope_strided_tokens_and_empty():
+    H, D, n, ld = 4, 64, 9, 4 * 64 * 3
+    buf = _randn((n, ld), "f32", 3)
+    pos = torch.arange(n).float() * 1.5
+    ref = buf.clone().numpy()
+    ref[:, :H * D] = oracle.rope(ref[:, :H * D].reshape(n, H, D).copy(), pos.numpy()).reshape(n, H * D)
+    bd = dev(buf)
+    sp.sp_rope_apply(bd, dev(pos), H, D, ld_token=ld)
+    np.testing.assert_allclose(f32(bd), ref, atol=4e-6)
+    sp.sp_rope_apply(bd, dev(pos), H, D, n_tokens=0)      # no-op
+
+
+# ------------------------------------------------------------------------- prefill
+def _prefill_gpu(q, k, v, lay, scale, rows=sp.SP_ROWS_ALL, poison=True):
+    dl = sp.DeviceLayout.from_host(lay)
+    T, H, D = q.shape
+    qd, kd, vd = dev(q), dev(k), dev(v)
+    out = torch.full_like(qd, float("nan")) if poison else torch.zeros_like(qd)
+    lse = torch.full((H, T), float("nan"), device="cuda")
+    ws = workspace(sp.sp_prefill_workspace_bytes(dl, H, D, sp.dtype_code(qd)))
+    sp.sp_superpose_prefill(qd, kd, vd, dl, scale, out, lse, ws, rows=rows)
+    sp.sp_check_status(ws)
+    return f32(out), lse.cpu().numpy()
+
+
+def _check_prefill(lay, H, Hkv, D, dtype, seed, std=1.0, scale=None):
+    T = lay.total_tokens
+    q = _randn((T, H, D), dtype, seed, std)
+    k = _randn((T, Hkv, D), dtype, seed + 1, std)
+    v = _randn((T, Hkv, D), dtype, seed + 2)
+    scale = 1 / math.sqrt(D) if scale is None else scale
+    ref_o, ref_l = oracle.prefill(f32(q), f32(k), f32(v), lay, scale)
+    got_o, got_l = _prefill_gpu(q, k, v, lay, scale)
+    assert not np.isnan(got_o).any(), "rows left unwritten"
+    assert rel_l2(got_o, ref_o) <= TOL[dtype]
+    np.testing.assert_allclose(got_l, ref_l, atol=1e-5 if dtype == "f32" else 2e-2)
+    # per-row check too, so that a single bad row cannot hide in the norm
+    num = np.linalg.norm((got_o - ref_o).reshape(T, -1), axis=1)
+    den = np.linalg.norm(ref_o.reshape(T, -1), axis=1) + 1e-6
+    assert (num / den).max() <= 5 * TOL[dtype]
+    return q, k, v, got_o, got_l
+
+
+@pytest.mark.parametrize("cfg", CONFIGS[:2], ids=lambda c: c.name)
+def test_prefill_config_full(cfg):
+    lay = draw_lengths(cfg)
+    q, k, v = draw_qkv(cfg, lay)
+    scale = 1 / math.sqrt(cfg.head_dim)
+    ref_o, ref_l = oracle.prefill(f32(q), f32(k), f32(v), lay, scale)
+    got_o, got_l = _prefill_gpu(q, k, v, lay, scale)
+    assert rel_l2(got_o, ref_o) <= TOL[cfg.dtype]
+    np.testing.assert_allclose(got_l, ref_l, atol=1e-5 if cfg.dtype == "f32" else 2e-2)
+
+
+@pytest.mark.parametrize("dtype,D", [("f32", 64), ("f32", 128), ("bf16", 64), ("bf16", 128)])
+def test_prefill_ragged_edges(dtype, D):
+    """Lengths around tile edges, empty preamble, empty documents, single rows."""
+    lay = build_layout([0, 5, 16, 130],
+                       [[1, 15, 16], [17, 127, 0], [128, 129], [300, 2, 64]],
+                       [[1, 1, 2], [3, 1, 8], [7, 24], [33, 1, 64]])
+    _check_prefill(lay, 4, 2, D, dtype, 100, std=1.0)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_prefill_peaky_scores_and_planted_keys(dtype):
+    """Unscaled N(0,1) q.k (sharp softmax) and one dominant key per row: masking or
+    rescaling mistakes cannot hide behind a near-uniform softmax."""
+    D, H = 128, 2
+    lay = build_layout([40], [[200, 77]], [[24, 24]])
+    _check_prefill(lay, H, H, D, dtype, 200, std=1.0, scale=0.35)
+    T = lay.total_tokens
+    q = _randn((T, H, D), dtype, 300, 0.05)
+    k = _randn((T, H, D), dtype, 301, 0.05)
+    v = _randn((T, H, D), dtype, 302)
+    g = np.random.default_rng(5)
+    for r in range(T):                      # plant: row r's query matches one allowed key strongly
+        c = int(g.integers(0, r + 1)) if r < 40 else int(g.integers(0, 40))
+        q[r] = (k[c].float() * 60).to(q.dtype)
+    ref_o, _ = oracle.prefill(f32(q), f32(k), f32(v), lay, 1.0)
+    got_o, _ = _prefill_gpu(q, k, v, lay, 1.0)
+    assert rel_l2(got_o, ref_o) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("dtype,D", [("f32", 64), ("bf16", 128)])
+def test_prefill_query_only_rows(dtype, D):
+    lay = build_layout([9, 33], [[50, 140], [7]], [[8, 8], [24]])
+    H = 2
+    T = lay.total_tokens
+    q, k, v = (_randn((T, H, D), dtype, s) for s in (11, 12, 13))
+    scale = 1 / math.sqrt(D)
+    ref_o, ref_l = oracle.prefill(f32(q), f32(k), f32(v), lay, scale)
+    got_o, got_l = _prefill_gpu(q, k, v, lay, scale, rows=sp.SP_ROWS_QUERY_ONLY)
+    is_q = np.zeros(T, bool)
+    for i in range(lay.n_paths):
+        s = lay.path_start[i] + lay.doc_len[i]
+        is_q[s:s + lay.qry_len[i]] = True
+    assert np.isnan(got_o[~is_q]).all(), "non-query rows must stay untouched"
+    assert rel_l2(got_o[is_q], ref_o[is_q]) <= TOL[dtype]
+    np.testing.assert_allclose(got_l[:, is_q], ref_l[:, is_q], atol=1e-5 if dtype == "f32" else 2e-2)
+
+
+def test_prefill_is_deterministic():
+    cfg = CONFIGS[1]
+    lay = draw_lengths(cfg)
+    q, k, v = draw_qkv(cfg, lay)
+    a, la = _prefill_gpu(q, k, v, lay, 0.0884)
+    b, lb = _prefill_gpu(q, k, v, lay, 0.0884)
+    np.testing.assert_array_equal(a, b)
+    np.testing.assert_array_equal(la, lb)
+
+
+# ------------------------------------------------------------------------- path scores
+def _scores_gpu(logits, tgt, off, prior, weight, with_rows=True):
+    R = logits.shape[0]
+    n_paths = len(off) - 1
+    scores = torch.full((n_paths,), float("nan"), device="cuda")
+    rows = torch.full((R,), float("nan"), device="cuda") if with_rows else None
+    ws = workspace(sp.sp_path_scores_workspace_bytes(R))
+    sp.sp_path_scores(dev(logits), dev(tgt), dev(off), scores,
+                      None if prior is None else dev(prior), None if weight is None else dev(weight),
+                      rows, ws)
+    return scores.cpu().numpy(), None if rows is None else rows.cpu().numpy()
+
+
+@pytest.mark.parametrize("cfg", CONFIGS[:2], ids=lambda c: c.name)
+def test_path_scores_config_full(cfg):
+    lay = draw_lengths(cfg)
+    logits = draw_logits(cfg, lay)
+    tgt = draw_targets(cfg, lay)
+    prior, weight = draw_prior_weight(cfg, lay)
+    off = lay.query_row_offsets()
+    ref_s, ref_r = oracle.path_scores(f32(logits), tgt, off, prior, weight)
+    got_s, got_r = _scores_gpu(logits, tgt, off, prior, weight)
+    np.testing.assert_allclose(got_r, ref_r, atol=1e-3)
+    sums_got = np.add.reduceat(got_r, off[:-1])
+    sums_ref = np.add.reduceat(ref_r, off[:-1])
+    assert np.all(np.abs(sums_got - sums_ref) <= 1e-3 * lay.qry_len)
+    assert np.all(np.abs(got_s - ref_s) <= 1e-3 * lay.qry_len * weight + 1e-6)
+    # reproducible bit for bit, with or without the row output
+    again, _ = _scores_gpu(logits, tgt, off, prior, weight, with_rows=False)
+    np.testing.assert_array_equal(got_s, again)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [1, 7, 8, 1000, 4099, 50432])
+def test_path_scores_vocab_edges(dtype, V):
+    qlens = [1, 3, 0, 5]
+    off = np.concatenate([[0], np.cumsum(qlens)]).astype(np.int32)
+    logits = _randn((int(off[-1]), V), dtype, 40 + V, 3.0)
+    g = np.random.default_rng(V)
+    tgt = g.integers(0, V, size=int(off[-1])).astype(np.int32)
+    tgt[[0, 3]] = -1
+    ref_s, ref_r = oracle.path_scores(f32(logits), tgt, off)
+    got_s, got_r = _scores_gpu(logits, tgt, off, None, None)
+    np.testing.assert_allclose(got_r, ref_r, atol=1e-4)
+    np.testing.assert_allclose(got_s, ref_s, atol=1e-3)
+    assert got_s[2] == 0.0                      # a path with no rows scores its prior (0)
+
+
+def test_path_scores_unaligned_rows_and_large_offsets():
+    V, ld = 1003, 1011                          # odd stride: rows are not 16-byte aligned
+    buf = _randn((6, ld), "bf16", 77, 3.0)
+    logits = buf[:, :V]
+    off = np.array([0, 6], np.int32)
+    tgt = np.array([5, 1002, 0, 17, -1, 400], np.int32)
+    ref_s, ref_r = oracle.path_scores(f32(logits), tgt, off)
+    scores = torch.zeros(1, device="cuda")
+    rows = torch.zeros(6, device="cuda")
+    sp.sp_path_scores(dev(buf)[:, :V], dev(tgt), dev(off), scores, row_logp=rows)
+    np.testing.assert_allclose(rows.cpu().numpy(), ref_r, atol=1e-4)
+    # logits far from zero: the running maximum must carry the scale
+    shifted = (f32(logits) * 0 + 3.0e4).astype(np.float32)
+    shifted[:, ::7] += 11.0
+    ref_s, ref_r = oracle.path_scores(shifted, tgt, off)
+    got_s, got_r = _scores_gpu(torch.from_numpy(shifted), tgt, off, None, None)
+    np.testing.assert_allclose(got_r, ref_r, atol=1e-3)
+
+
+# ------------------------------------------------------------------------- top-k
+def _topk_gpu(scores, ppo, k):
+    B = len(ppo) - 1
+    idx = torch.full((B, k), -7, dtype=torch.int32, device="cuda")
+    post = torch.full((B, k), float("nan"), device="cuda")
+    sp.sp_prune_topk(dev(scores), dev(ppo), k, idx, post)
+    return idx.cpu().numpy(), post.cpu().numpy()
+
+
+@pytest.mark.parametrize("n,k", [(4, 1), (20, 2), (100, 4), (400, 8), (33, 33), (5, 9), (1000, 64)])
+def test_topk_bit_exact(n, k):
+    g = np.random.default_rng(n * 31 + k)
+    ppo = np.array([0, n, n, 2 * n + 3], np.int32)
+    s = g.standard_normal(int(ppo[-1])).astype(np.float32)
+    s[g.integers(0, len(s), size=len(s) // 4)] = s[0]        # many exact ties
+    ref_i, ref_p = oracle.prune_topk(s, ppo, k)
+    got_i, got_p = _topk_gpu(s, ppo, k)
+    np.testing.assert_array_equal(got_i, ref_i)
+    np.testing.assert_allclose(got_p, ref_p, rtol=2e-5, atol=1e-9)
+
+
+def test_topk_nan_inf_and_signed_zero():
+    ppo = np.array([0, 8, 12], np.int32)
+    s = np.array([0.0, -0.0, np.nan, np.inf, -np.inf, 1.0, np.nan, 0.0,
+                  np.nan, np.nan, -np.inf, -np.inf], np.float32)
+    ref_i, ref_p = oracle.prune_topk(s[:8].copy(), ppo[:2], 8)
+    got_i, got_p = _topk_gpu(s, ppo, 8)
+    np.testing.assert_array_equal(got_i[0], ref_i[0])
+    assert list(got_i[0]) == [3, 5, 0, 1, 7, 4, 2, 6]
+    ref_i2, ref_p2 = oracle.prune_topk(s, ppo, 8)
+    np.testing.assert_array_equal(got_i, ref_i2)
+    np.testing.assert_array_equal(got_p[1], ref_p2[1])           # all -inf / NaN: posterior 0
+
+
+# ------------------------------------------------------------------------- decode
+def _decode_case(lay, H, Hkv, D, dtype, k, kept, tail_cap, tail_len, seed, scale=None, std=1.0):
+    B, T = lay.n_prompts, lay.total_tokens
+    kc = _randn((T, Hkv, D), dtype, seed, std)
+    vc = _randn((T, Hkv, D), dtype, seed + 1)
+    q = _randn((B, H, D), dtype, seed + 2, std)
+    tk = _randn((B, max(tail_cap, 1), Hkv, D), dtype, seed + 3, std)
+    tv = _randn((B, max(tail_cap, 1), Hkv, D), dtype, seed + 4)
+    scale = 1 / math.sqrt(D) if scale is None else scale
+    kept = np.asarray(kept, np.int32).reshape(B, k)
+    tl = np.asarray(tail_len, np.int32)
+    ref_o, ref_l = oracle.pruned_decode(f32(q), f32(kc), f32(vc), lay, kept, f32(tk), f32(tv), tl, scale)
+    dl = sp.DeviceLayout.from_host(lay)
+    out = torch.full((B, H, D), float("nan"), dtype=TDT[dtype], device="cuda")
+    lse = torch.full((B, H), float("nan"), device="cuda")
+    ws = workspace(sp.sp_decode_workspace_bytes(B, H, D))
+    args = (dev(q), dev(kc), dev(vc), dl, dev(kept), k,
+            dev(tk) if tail_cap else None, dev(tv) if tail_cap else None, dev(tl) if tail_cap else None,
+            tail_cap, scale, out, lse, ws)
+    sp.sp_pruned_decode(*args)
+    sp.sp_check_status(ws)
+    got_o, got_l = f32(out), lse.cpu().numpy()
+    assert rel_l2(got_o, ref_o) <= TOL[dtype]
+    fin = np.isfinite(ref_l)
+    np.testing.assert_allclose(got_l[fin], ref_l[fin], atol=1e-5 if dtype == "f32" else 2e-2)
+    np.testing.assert_array_equal(got_l[~fin], ref_l[~fin])
+    out2 = torch.full_like(out, float("nan"))
+    sp.sp_pruned_decode(*args[:11], out2, lse, ws)      # same workspace again: bit-identical
+    np.testing.assert_array_equal(f32(out2), got_o)
+    return got_o
+
+
+@pytest.mark.parametrize("dtype,D", [("f32", 64), ("f32", 128), ("bf16", 64), ("bf16", 128)])
+def test_decode_small_batches_split_kv(dtype, D):
+    lay = build_layout([16, 3], [[32, 1, 129, 40], [200, 17]], [[8, 8, 8, 8], [5, 5]])
+    _decode_case(lay, 4, 2, D, dtype, 2, [[2, 0], [4, -1]], 6, [6, 1], 500)
+    _decode_case(lay, 4, 4, D, dtype, 4, [[3, 2, 1, 0], [5, 4, -1, -1]], 0, [0, 0], 510)   # k = N, no tail
+    _decode_case(lay, 2, 1, D, dtype, 1, [[-1], [-1]], 3, [0, 2], 520)                     # nothing kept
+
+
+def test_decode_no_keys_at_all():
+    lay = build_layout([0, 4], [[5], [6]], [[2], [2]])
+    got = _decode_case(lay, 2, 2, 64, "f32", 1, [[-1], [1]], 2, [0, 1], 530)
+    assert np.all(got[0] == 0.0)
+
+
+@pytest.mark.parametrize("cfg", CONFIGS[:2], ids=lambda c: c.name)
+def test_decode_config_steps(cfg):
+    """The config's decode loop: kept paths from the oracle's top-k, tail growing by one
+    token per step (the new token attends to itself)."""
+    lay = draw_lengths(cfg)
+    _, kc, vc = draw_qkv(cfg, lay)
+    steps = min(cfg.decode_steps, 5)
+    q, tk, tv = draw_decode_inputs(cfg, lay.n_prompts, steps)
+    scores = np.random.default_rng(cfg.seed).standard_normal(lay.n_paths).astype(np.float32)
+    kept, _ = oracle.prune_topk(scores, lay.prompt_path_off, cfg.top_k)
+    dl = sp.DeviceLayout.from_host(lay)
+    B, H, D = lay.n_prompts, cfg.n_heads, cfg.head_dim
+    ws = workspace(sp.sp_decode_workspace_bytes(B, H, D))
+    kcd, vcd, tkd, tvd, keptd = dev(kc), dev(vc), dev(tk), dev(tv), dev(kept)
+    scale = 1 / math.sqrt(D)
+    for t in range(steps):
+        tl = np.full(B, t + 1, np.int32)
+        ref_o, _ = oracle.pruned_decode(f32(q[t]), f32(kc), f32(vc), lay, kept, f32(tk), f32(tv), tl, scale)
+        out = torch.empty((B, H, D), dtype=TDT[cfg.dtype], device="cuda")
+        sp.sp_pruned_decode(dev(q[t]), kcd, vcd, dl, keptd, cfg.top_k, tkd, tvd, dev(tl), steps, scale, out, None, ws)
+        assert rel_l2(f32(out), ref_o) <= TOL[cfg.dtype]
+
+
+# ------------------------------------------------------------------------- whole chain
+@pytest.mark.parametrize("cfg", CONFIGS[:2], ids=lambda c: c.name)
+def test_chain_rope_prefill_scores_topk_decode(cfg):
+    """One pass of the hot path, each stage fed by the previous stage's device output,
+    against the same chain in the oracle."""
+    lay = draw_lengths(cfg)
+    B, H, Hkv, D = lay.n_prompts, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim
+    q, k, v = draw_qkv(cfg, lay)
+    if cfg.positions == "equilibrium":
+        pos, nxt = positions_for(lay, lambda P, L, Q: sp.sp_positions(P, L, Q))
+        pos_ref, _ = positions_for(lay, lambda P, L, Q: oracle.positions(P, L, Q))
+    else:
+        pos, nxt = positions_for(lay, lambda P, L, Q: sp.sp_positions(P, L, Q, scheme=sp.SP_POS_LEFT_ALIGNED))
+        pos_ref, _ = positions_for(lay, lambda P, L, Q: oracle.positions(P, L, Q, scheme="left"))
+    np.testing.assert_array_equal(pos, pos_ref)
+    scale = 1 / math.sqrt(D)
+    dl = sp.DeviceLayout.from_host(lay)
+    qd, kd, vd, posd = dev(q), dev(k), dev(v), dev(pos)
+    sp.sp_rope_apply(qd, posd, H, D, base=cfg.rope_base)
+    sp.sp_rope_apply(kd, posd, Hkv, D, base=cfg.rope_base)
+    out = torch.empty_like(qd)
+    ws = workspace(sp.sp_prefill_workspace_bytes(dl, H, D, sp.dtype_code(qd)))
+    sp.sp_superpose_prefill(qd, kd, vd, dl, scale, out, None, ws)
+    # oracle chain (rounding the rotated tensors to the storage type, as the device does)
+    rnd = (lambda a: a) if cfg.dtype == "f32" else (lambda a: torch.from_numpy(a).bfloat16().float().numpy())
+    q_r = rnd(oracle.rope(f32(q), pos_ref, base=cfg.rope_base))
+    k_r = rnd(oracle.rope(f32(k), pos_ref, base=cfg.rope_base))
+    ref_o, _ = oracle.prefill(q_r, k_r, f32(v), lay, scale)
+    assert rel_l2(f32(out), ref_o) <= TOL[cfg.dtype] * (1 if cfg.dtype == "bf16" else 3)
+
+    logits, tgt = draw_logits(cfg, lay), draw_targets(cfg, lay)
+    prior, weight = draw_prior_weight(cfg, lay)
+    off = lay.query_row_offsets()
+    scores = torch.empty(lay.n_paths, device="cuda")
+    ws2 = workspace(sp.sp_path_scores_workspace_bytes(logits.shape[0]))
+    sp.sp_path_scores(dev(logits), dev(tgt), dev(off), scores, dev(prior), dev(weight), None, ws2)
+    kept = torch.empty((B, cfg.top_k), dtype=torch.int32, device="cuda")
+    post = torch.empty((B, cfg.top_k), device="cuda")
+    sp.sp_prune_topk(scores, dl.prompt_path_off, cfg.top_k, kept, post)
+    ref_s, _ = oracle.path_scores(f32(logits), tgt, off, prior, weight)
+    ref_kept, ref_post = oracle.prune_topk(ref_s, lay.prompt_path_off, cfg.top_k)
+    tol = 1e-3 * cfg.qry_len * float(weight.max())
+    for b in range(B):       # bit-exact where the k-th / (k+1)-th gap exceeds twice the tolerance
+        lo, hi = lay.prompt_path_off[b], lay.prompt_path_off[b + 1]
+        srt = np.sort(ref_s[lo:hi])[::-1]
+        gaps = np.abs(np.diff(srt[:cfg.top_k + 1]))
+        if gaps.size == 0 or gaps.min() > 2 * tol:
+            np.testing.assert_array_equal(kept[b].cpu().numpy(), ref_kept[b])
+        else:
+            assert set(kept[b].cpu().numpy()) <= set(np.where(ref_s[lo:hi] >= srt[cfg.top_k - 1] - 2 * tol)[0] + lo)
+    np.testing.assert_allclose(post.cpu().numpy(), ref_post, rtol=5e-3, atol=1e-6)
+
+    steps = 3
+    dq, tk, tv = draw_decode_inputs(cfg, B, steps)
+    tkd, tvd = dev(tk), dev(tv)
+    ws3 = workspace(sp.sp_decode_workspace_bytes(B, H, D))
+    kept_h = kept.cpu().numpy()
+    tk_ref, tv_ref = f32(tk).copy(), f32(tv)
+    for t in range(steps):
+        tpos = np.asarray(nxt + t, np.float32)          # task / response positions continue with step 1
+        qt = dev(dq[t])
+        sp.sp_rope_apply(qt, dev(tpos), H, D, base=cfg.rope_base)
+        sp.sp_rope_apply(tkd[:, t], dev(tpos), Hkv, D, n_tokens=B, ld_token=steps * Hkv * D, base=cfg.rope_base)
+        o = torch.empty((B, H, D), dtype=TDT[cfg.dtype], device="cuda")
+        tl = np.full(B, t + 1, np.int32)
+        sp.sp_pruned_decode(qt, kd, vd, dl, kept, cfg.top_k, tkd, tvd, dev(tl), steps, scale, o, None, ws3)
+        qt_ref = rnd(oracle.rope(f32(dq[t]), tpos, base=cfg.rope_base))
+        tk_ref[:, t] = rnd(oracle.rope(np.ascontiguousarray(tk_ref[:, t]), tpos, base=cfg.rope_base))
+        ref_d, _ = oracle.pruned_decode(qt_ref, k_r, f32(v), lay, kept_h, tk_ref, tv_ref, tl, scale)
+        assert rel_l2(f32(o), ref_d) <= TOL[cfg.dtype] * (1 if cfg.dtype == "bf16" else 3)
