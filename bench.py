@@ -1,0 +1,431 @@
+#!/usr/bin/env python
+"""Benchmark of the superposition-prompting hot path on B200.
+
+One "step" is one pass of the whole path over one batch of synthetic prompts:
+  RoPE(Q), RoPE(K) -> fork-join prefill -> path scores -> top-k -> decode_steps x
+  (RoPE of the new q and k rows, pruned decode).
+`value` is the prefill's useful TFLOP/s counted over the WHOLE step time (inputs resident
+in HBM); the per-kernel rates and roofline fractions are reported beside it.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+N > 1 (torchrun): every rank runs its own batch (independent prompts, no data-path
+collective); the time is the max over ranks and `value` the aggregate ("weak" scaling).
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import (draw_decode_inputs, draw_lengths, draw_logits, draw_prior_weight,  # noqa: E402
+                       draw_qkv, draw_targets, get_config)
+
+METRIC = "superposition prefill useful TFLOP/s over the whole hot-path step"
+UNIT = "TFLOP/s"
+PREFILL_LAUNCHES = 1           # kernels sp_superpose_prefill launches per call
+# dram__bytes_read.sum + dram__bytes_write.sum of one prefill launch, from the ncu capture
+# summarised under profiles/ (None until captured for the current kernel).
+NCU_PREFILL_TRAFFIC_BYTES = {}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+def positions_all(lay, fn):
+    pos = np.zeros(lay.total_tokens, dtype=np.float32)
+    nxt = np.zeros(lay.n_prompts, dtype=np.float64)
+    for b in range(lay.n_prompts):
+        p0, p1 = int(lay.prompt_path_off[b]), int(lay.prompt_path_off[b + 1])
+        q = int(lay.qry_len[p0]) if p1 > p0 else 0
+        p, _, n = fn(int(lay.pre_len[b]), lay.doc_len[p0:p1], q)
+        lo, hi = lay.prompt_row_range(b)
+        pos[lo:hi] = p
+        nxt[b] = n
+    return pos, nxt
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, pw = [], [], set(), []
+        for ln in list(self.lines):
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------
+class HotPath:
+    """Device buffers and the launch sequence of one step, through the C-ABI binding."""
+
+    def __init__(self, cfg, seed, sp, device):
+        self.cfg, self.sp = cfg, sp
+        t0 = time.time()
+        self.lay = lay = draw_lengths(cfg, seed=seed)
+        B, H, Hkv, D = lay.n_prompts, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim
+        self.B, self.H, self.Hkv, self.D = B, H, Hkv, D
+        self.tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+        self.steps_dec = cfg.decode_steps
+        # host inputs (pinned: they are also the source of the end-to-end copies)
+        self.h_q, self.h_k, self.h_v = draw_qkv(cfg, lay, seed=seed, pin=True)
+        self.h_logits = draw_logits(cfg, lay, seed=seed, pin=True)
+        self.h_tgt = torch.from_numpy(draw_targets(cfg, lay, seed=seed)).pin_memory()
+        prior, weight = draw_prior_weight(cfg, lay, seed=seed)
+        self.h_dq, self.h_tk, self.h_tv = draw_decode_inputs(cfg, B, self.steps_dec, seed=seed, pin=True)
+        scheme = sp.SP_POS_EQUILIBRIUM if cfg.positions == "equilibrium" else sp.SP_POS_LEFT_ALIGNED
+        pos, nxt = positions_all(lay, lambda P, L, Q: sp.sp_positions(P, L, Q, scheme=scheme))
+        self.h_pos = torch.from_numpy(pos).pin_memory()
+        tpos = (nxt[None, :] + np.arange(self.steps_dec)[:, None]).astype(np.float32)   # [steps, B]
+        self.gen_s = time.time() - t0
+
+        dv = lambda t: t.to(device, non_blocking=True)
+        self.dl = sp.DeviceLayout.from_host(lay, device)
+        self.q, self.k, self.v = dv(self.h_q), dv(self.h_k), dv(self.h_v)
+        self.out = torch.empty_like(self.q)
+        self.logits, self.tgt, self.pos = dv(self.h_logits), dv(self.h_tgt), dv(self.h_pos)
+        self.row_off = torch.from_numpy(lay.query_row_offsets()).to(device)
+        self.prior, self.weight = torch.from_numpy(prior).to(device), torch.from_numpy(weight).to(device)
+        self.scores = torch.empty(lay.n_paths, device=device)
+        self.kept = torch.empty((B, cfg.top_k), dtype=torch.int32, device=device)
+        self.post = torch.empty((B, cfg.top_k), device=device)
+        self.dq, self.tk, self.tv = dv(self.h_dq), dv(self.h_tk), dv(self.h_tv)
+        self.tpos = torch.from_numpy(tpos).to(device)
+        self.tail_len = (torch.arange(1, self.steps_dec + 1, dtype=torch.int32)[:, None]
+                         .expand(self.steps_dec, B).contiguous().to(device))
+        self.dec_out = torch.empty((self.steps_dec, B, H, D), dtype=self.tdt, device=device)
+        ws = lambda n: torch.zeros(max(int(n), 256), dtype=torch.uint8, device=device)
+        self.ws_pre = ws(sp.sp_prefill_workspace_bytes(self.dl, H, D, sp.dtype_code(self.q)))
+        self.ws_sc = ws(sp.sp_path_scores_workspace_bytes(self.logits.shape[0]))
+        self.ws_dec = ws(sp.sp_decode_workspace_bytes(B, H, D))
+        self.scale = 1.0 / math.sqrt(D)
+        self.h_dec_out = torch.empty(self.dec_out.shape, dtype=self.tdt).pin_memory()
+        self.h_kept = torch.empty(self.kept.shape, dtype=torch.int32).pin_memory()
+        torch.cuda.synchronize()
+
+        # algorithmic work per step
+        eb = cfg.elt_bytes
+        T = lay.total_tokens
+        self.pairs = lay.allowed_pairs()
+        self.flop_prefill = 4.0 * D * H * self.pairs
+        self.bytes_prefill = float(T) * (2 * H + 2 * Hkv) * D * eb
+        self.bytes_rope = 2.0 * T * (H + Hkv) * D * eb
+        scored = int((self.h_tgt >= 0).sum())
+        self.bytes_scores = float(scored) * cfg.vocab * eb
+        self.bytes_decode = None        # needs the kept set: filled after the first step
+        # kernels launched per step (ours): rope x2, prefill, row_logp + path_sum, top-k,
+        # per decode step rope x2 + decode
+        self.launches = 2 + PREFILL_LAUNCHES + 2 + 1 + self.steps_dec * 3
+
+    def decode_bytes(self):
+        kept = self.kept.cpu().numpy()
+        lay = self.lay
+        tot = 0
+        for b in range(self.B):
+            n = int(lay.pre_len[b]) + sum(int(lay.doc_len[i] + lay.qry_len[i]) for i in kept[b] if i >= 0)
+            tot += sum(n + t + 1 for t in range(self.steps_dec))
+        return float(tot) * 2 * self.Hkv * self.D * self.cfg.elt_bytes
+
+    def h2d(self):
+        nb = 0
+        for d, h in ((self.q, self.h_q), (self.k, self.h_k), (self.v, self.h_v), (self.logits, self.h_logits),
+                     (self.tgt, self.h_tgt), (self.pos, self.h_pos), (self.dq, self.h_dq), (self.tk, self.h_tk),
+                     (self.tv, self.h_tv)):
+            d.copy_(h, non_blocking=True)
+            nb += h.numel() * h.element_size()
+        return nb
+
+    def d2h(self):
+        self.h_dec_out.copy_(self.dec_out, non_blocking=True)
+        self.h_kept.copy_(self.kept, non_blocking=True)
+        return self.h_dec_out.numel() * self.h_dec_out.element_size() + self.h_kept.numel() * 4
+
+    def step(self, ev=None):
+        """Launches one pass.  ev (optional): list that receives CUDA events at stage edges."""
+        sp, cfg = self.sp, self.cfg
+        H, Hkv, D, B = self.H, self.Hkv, self.D, self.B
+        mark = (lambda: None) if ev is None else (lambda: (ev.append(torch.cuda.Event(enable_timing=True)), ev[-1].record()))
+        mark()
+        sp.sp_rope_apply(self.q, self.pos, H, D, base=cfg.rope_base)
+        sp.sp_rope_apply(self.k, self.pos, Hkv, D, base=cfg.rope_base)
+        mark()
+        sp.sp_superpose_prefill(self.q, self.k, self.v, self.dl, self.scale, self.out, None, self.ws_pre)
+        mark()
+        sp.sp_path_scores(self.logits, self.tgt, self.row_off, self.scores, self.prior, self.weight, None, self.ws_sc)
+        mark()
+        sp.sp_prune_topk(self.scores, self.dl.prompt_path_off, cfg.top_k, self.kept, self.post)
+        mark()
+        ld = self.steps_dec * Hkv * D
+        for t in range(self.steps_dec):
+            sp.sp_rope_apply(self.dq[t], self.tpos[t], H, D, base=cfg.rope_base)
+            sp.sp_rope_apply(self.tk[:, t], self.tpos[t], Hkv, D, n_tokens=B, ld_token=ld, base=cfg.rope_base)
+            sp.sp_pruned_decode(self.dq[t], self.k, self.v, self.dl, self.kept, cfg.top_k, self.tk, self.tv,
+                                self.tail_len[t], self.steps_dec, self.scale, self.dec_out[t], None, self.ws_dec)
+        mark()
+
+
+STAGES = ("rope", "prefill", "path_scores", "topk", "decode")
+
+
+def run_ours(args):
+    import paper_2404_06910_b200 as sp          # raises if the CUDA library is missing
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    cfg = get_config(args.workload)
+    hp = HotPath(cfg, cfg.seed + 1000 * rank, sp, device)
+    peaks = load_peaks()
+    l2_bytes = torch.cuda.get_device_properties(device).L2_cache_size
+    flush = None
+    if hp.bytes_prefill < 2 * l2_bytes:          # small workload: flush L2 between steps
+        flush = torch.empty(2 * l2_bytes, dtype=torch.uint8, device=device)
+
+    def sync():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        hp.step()
+        if flush is not None:
+            flush.zero_()
+    sync()
+    hp.bytes_decode = hp.decode_bytes()
+
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else 0)
+    if rank == 0:
+        sampler.start()
+    all_ev = []
+    sync()
+    for _ in range(args.steps):
+        ev = []
+        hp.step(ev)
+        all_ev.append(ev)
+        if flush is not None:
+            flush.zero_()
+    sync()
+    clocks = sampler.stop() if rank == 0 else None
+
+    stage_ms = np.zeros(len(STAGES))
+    total_ms = 0.0
+    for ev in all_ev:
+        for i in range(len(STAGES)):
+            stage_ms[i] += ev[i].elapsed_time(ev[i + 1])
+        total_ms += ev[0].elapsed_time(ev[-1])
+    stage_ms /= args.steps
+    ms_per_step = total_ms / args.steps
+
+    # end to end: pinned host -> device copies of every input, the pass, device -> host results
+    e2e_steps = max(1, min(args.steps, 3))
+    hp.h2d(); hp.step(); hp.d2h(); sync()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        bi = hp.h2d()
+        hp.step()
+        bo = hp.d2h()
+    e1.record()
+    sync()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    t = torch.tensor([ms_per_step, e2e_ms], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_per_step, e2e_ms = float(t[0]), float(t[1])
+
+    if rank == 0:
+        tf = lambda flop, ms: flop / (ms * 1e-3) / 1e12
+        gb = lambda byt, ms: byt / (ms * 1e-3) / 1e9
+        ms = dict(zip(STAGES, stage_ms))
+        pre_gbs, pre_tf = gb(hp.bytes_prefill, ms["prefill"]), tf(hp.flop_prefill, ms["prefill"])
+        ai = hp.flop_prefill / hp.bytes_prefill
+        bound_tf = min(peaks["bf16_tflops_sustained"], ai * peaks["hbm_gbs"] / 1e3)
+        kernels = {
+            "rope": {"ms": ms["rope"], "gbs": gb(hp.bytes_rope, ms["rope"]), "frac_hbm": gb(hp.bytes_rope, ms["rope"]) / peaks["hbm_gbs"]},
+            "prefill": {"ms": ms["prefill"], "useful_tflops": pre_tf, "gbs": pre_gbs,
+                        "frac_bf16_burst": pre_tf / peaks["bf16_tflops"],
+                        "frac_bf16_sustained": pre_tf / peaks["bf16_tflops_sustained"],
+                        "arith_intensity": ai, "binding_roofline_tflops": bound_tf, "frac_binding": pre_tf / bound_tf},
+            "path_scores": {"ms": ms["path_scores"], "gbs": gb(hp.bytes_scores, ms["path_scores"]),
+                            "frac_hbm": gb(hp.bytes_scores, ms["path_scores"]) / peaks["hbm_gbs"]},
+            "topk": {"ms": ms["topk"]},
+            "decode": {"ms": ms["decode"], "steps": hp.steps_dec, "gbs": gb(hp.bytes_decode, ms["decode"]),
+                       "frac_hbm": gb(hp.bytes_decode, ms["decode"]) / peaks["hbm_gbs"],
+                       "includes": "2 rope launches + 1 decode launch per token"},
+        }
+        line = {
+            "metric": METRIC, "value": world * tf(hp.flop_prefill, ms_per_step), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": cfg.name, "prompts_per_gpu": hp.B, "paths": hp.lay.n_paths,
+                       "tokens": hp.lay.total_tokens, "heads": hp.H, "head_dim": hp.D, "vocab": cfg.vocab,
+                       "top_k": cfg.top_k, "decode_steps": hp.steps_dec, "allowed_pairs": hp.pairs,
+                       "l2": "inputs larger than L2" if flush is None else "L2 flushed between steps",
+                       "parallelism": f"dp{world} (independent prompts per GPU, no collective)"},
+            "roofline": {"kernel": "sp_superpose_prefill", "bound": "hbm", "achieved": pre_gbs,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": pre_gbs / peaks["hbm_gbs"],
+                         "traffic": NCU_PREFILL_TRAFFIC_BYTES.get(cfg.name), "peak_source": peaks["source"],
+                         "algorithmic_bytes": hp.bytes_prefill, "useful_tflops": pre_tf,
+                         "frac_bf16_sustained": pre_tf / peaks["bf16_tflops_sustained"]},
+            "kernels": kernels,
+            "e2e": {"value": world * tf(hp.flop_prefill, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
+                    "steps": e2e_steps, "h2d_bytes_per_step": bi, "d2h_bytes_per_step": bo},
+            "gpu_launches": hp.launches * args.steps,
+            "clocks": clocks,
+            "input_generation_s": hp.gen_s,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(cfg, steps=1, warmup=0, budget_s=25.0)[0]
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------
+def oracle_sample_pass(cfg, n_paths):
+    """Returns a closure running the whole hot path in the CPU oracle on the first n_paths
+    paths of prompt 0 of the workload, and the useful prefill FLOPs of that sample."""
+    import oracle
+    from workloads import build_layout
+    from workloads.tensors import to_f32_numpy
+    full = draw_lengths(cfg)
+    n_paths = min(n_paths, int(full.prompt_path_off[1]))
+    lay = build_layout([int(full.pre_len[0])], [full.doc_len[:n_paths]], [full.qry_len[:n_paths]])
+    q, k, v = (to_f32_numpy(t) for t in draw_qkv(cfg, lay))
+    logits = to_f32_numpy(draw_logits(cfg, lay))
+    tgt = draw_targets(cfg, lay)
+    prior, weight = draw_prior_weight(cfg, lay)
+    steps = cfg.decode_steps
+    dq, tk, tv = (to_f32_numpy(t) for t in draw_decode_inputs(cfg, 1, steps))
+    scheme = "equilibrium" if cfg.positions == "equilibrium" else "left"
+    scale = 1.0 / math.sqrt(cfg.head_dim)
+    kk = min(cfg.top_k, n_paths)
+
+    def run():
+        pos, _, nxt = oracle.positions(int(lay.pre_len[0]), lay.doc_len, int(lay.qry_len[0]), scheme=scheme)
+        pos = pos.astype(np.float32)
+        qr = oracle.rope(q, pos, base=cfg.rope_base)
+        kr = oracle.rope(k, pos, base=cfg.rope_base)
+        oracle.prefill(qr, kr, v, lay, scale)
+        s, _ = oracle.path_scores(logits, tgt, lay.query_row_offsets(), prior, weight)
+        kept, _ = oracle.prune_topk(s, lay.prompt_path_off, kk)
+        tkr = tk.copy()
+        for t in range(steps):
+            tp = np.array([nxt + t], np.float32)
+            qt = oracle.rope(dq[t], tp, base=cfg.rope_base)
+            tkr[:, t] = oracle.rope(np.ascontiguousarray(tkr[:, t]), tp, base=cfg.rope_base)
+            oracle.pruned_decode(qt, kr, v, lay, kept, tkr, tv, np.array([t + 1], np.int32), scale)
+
+    flop = 4.0 * cfg.head_dim * cfg.n_heads * lay.allowed_pairs()
+    return run, flop, n_paths
+
+
+def cpu_baseline(cfg, steps, warmup, budget_s):
+    import oracle
+    n_paths = int(max(1, min(cfg.n_docs, (budget_s / max(1, steps + warmup)) // 0.4)))
+    run, flop, n_paths = oracle_sample_pass(cfg, n_paths)
+    for _ in range(warmup):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        run()
+    dt = (time.perf_counter() - t0) / steps
+    return ({"value": flop / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+             "sample": f"whole hot path on prompt 0 restricted to its first {n_paths} paths "
+                       f"({cfg.name}, all heads, {cfg.decode_steps} decode steps)",
+             "ms_per_sample": dt * 1e3}, dt)
+
+
+def run_reference(args):
+    """Times the CPU oracle (as it stands) on the host cores; rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    cfg = get_config(args.workload)
+    base, dt = cpu_baseline(cfg, args.steps, args.warmup, budget_s=150.0)
+    line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT,
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": {"workload": cfg.name, "sample": base["sample"]},
+            "cpu_baseline": base,
+            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
