@@ -179,6 +179,37 @@ int sp_pruned_decode(const void *q, const void *k_cache, const void *v_cache,
                      void *stream);
 
 /*
+ * Decode attention without a caller workspace.  (The paper has no counterpart: this entry
+ * point exists for integration reasons only.)  It computes exactly what sp_pruned_decode
+ * computes, with the same arguments minus (ws, ws_bytes), for callers that are not able to
+ * obtain device memory at the point of the call: code running inside a serving engine
+ * whose memory pool is fully handed out, plugins that are forbidden to call the CUDA
+ * allocator, or call sites where an allocation would stall the pipeline.  The split-KV
+ * scratch (arrival counters and per-split partial results) lives in one fixed
+ * 8 MiB array that is part of the library image; every GPU on which the library is used
+ * holds that array from load until the process exits.
+ *  - Limit: n_prompts*n_heads*4 bytes of counters (rounded up to 256) plus, when the key
+ *    sequence is split, n_prompts*n_heads*n_splits*(head_dim+2)*4 bytes of partials must
+ *    fit in sp_pruned_decode_static_max_bytes(); otherwise SP_ERR_WORKSPACE is returned and
+ *    nothing is launched (use sp_pruned_decode with your own workspace then).
+ *  - The call allocates and frees nothing.  The first call on each device looks up the
+ *    array's device address (a one-time runtime query made with that device current);
+ *    make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps whatever the previous call
+ *    left in it; each call clears the counters it needs on `stream` first.  Two calls
+ *    whose kernels can overlap on the GPU (different streams, no ordering between them)
+ *    race on the array: order them, or give one of them sp_pruned_decode and a workspace.
+ *  - No device status word is kept for this variant.
+ */
+size_t sp_pruned_decode_static_max_bytes(void);
+int sp_pruned_decode_static(const void *q, const void *k_cache, const void *v_cache,
+                            const sp_layout *lay, const int32_t *kept_idx, int k,
+                            const void *tail_k, const void *tail_v, const int32_t *tail_len,
+                            int tail_cap, int64_t max_keys, int n_heads, int n_kv_heads,
+                            int head_dim, float scale, void *out, float *lse, int dtype,
+                            void *stream);
+
+/*
  * Reads the device status word at the start of a workspace after synchronising `stream`.
  * Returns SP_OK, SP_ERR_TIMEOUT (a bounded wait expired; the outputs of that call are
  * not valid) or SP_ERR_CUDA.  The word is cleared by the next call that uses the workspace.

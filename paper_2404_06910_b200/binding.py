@@ -28,6 +28,7 @@ EXPORTS = (
     "sp_prefill_workspace_bytes", "sp_superpose_prefill",
     "sp_path_scores_workspace_bytes", "sp_path_scores", "sp_prune_topk",
     "sp_decode_workspace_bytes", "sp_pruned_decode", "sp_check_status",
+    "sp_pruned_decode_static_max_bytes", "sp_pruned_decode_static",
 )
 
 
@@ -73,6 +74,9 @@ def _load() -> ctypes.CDLL:
     lib.sp_pruned_decode.argtypes = [vp, vp, vp, lp, vp, c_int, vp, vp, vp, c_int, c_i64, c_int, c_int, c_int,
                                      c_f, vp, vp, vp, sz, c_int, vp]
     lib.sp_check_status.argtypes = [vp, vp]
+    lib.sp_pruned_decode_static_max_bytes.restype = sz
+    lib.sp_pruned_decode_static.argtypes = [vp, vp, vp, lp, vp, c_int, vp, vp, vp, c_int, c_i64, c_int, c_int, c_int,
+                                            c_f, vp, vp, c_int, vp]
     for name in EXPORTS:
         getattr(lib, name)          # raises AttributeError if a declared symbol is not exported
     return lib
@@ -203,6 +207,21 @@ def sp_pruned_decode(q, k_cache, v_cache, lay: DeviceLayout, kept_idx, k: int, t
     _check(lib.sp_pruned_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), ctypes.byref(lay.c), _ptr(kept_idx), k,
                                 _ptr(tail_k), _ptr(tail_v), _ptr(tail_len), tail_cap, max_keys, H, Hkv, D, scale,
                                 _ptr(out), _ptr(lse), _ptr(ws), _nbytes(ws), dtype_code(q), _stream(stream)))
+
+
+def sp_pruned_decode_static_max_bytes() -> int:
+    return int(lib.sp_pruned_decode_static_max_bytes())
+
+
+def sp_pruned_decode_static(q, k_cache, v_cache, lay: DeviceLayout, kept_idx, k: int, tail_k, tail_v, tail_len,
+                            tail_cap: int, scale: float, out, lse=None, max_keys: int = 0, stream=None):
+    """sp_pruned_decode for callers that cannot provide a workspace: the split-KV scratch is a
+    fixed array inside the library (see include/sp.h for its limit and sharing rules)."""
+    B, H, D = q.shape
+    Hkv = k_cache.shape[1]
+    _check(lib.sp_pruned_decode_static(_ptr(q), _ptr(k_cache), _ptr(v_cache), ctypes.byref(lay.c), _ptr(kept_idx),
+                                       k, _ptr(tail_k), _ptr(tail_v), _ptr(tail_len), tail_cap, max_keys, H, Hkv,
+                                       D, scale, _ptr(out), _ptr(lse), dtype_code(q), _stream(stream)))
 
 
 def sp_check_status(ws, stream=None) -> None:

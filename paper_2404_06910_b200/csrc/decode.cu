@@ -293,3 +293,100 @@ extern "C" int sp_pruned_decode(const void *q, const void *k_cache, const void *
     return head_dim == 128 ? launch_decode<float, 128>(a, lay->n_prompts, st)
                            : launch_decode<float, 64>(a, lay->n_prompts, st);
 }
+
+// ---------------------------------------------------------------------------------------
+// sp_pruned_decode_static: the same decode kernel for callers that have no device
+// allocator to ask for a workspace (see sp.h).  Its split-KV scratch (arrival counters and
+// per-split partial results) lives in one fixed array inside the library image.
+// ---------------------------------------------------------------------------------------
+namespace sp {
+
+constexpr size_t kStaticScratchBytes = 8u << 20;     // 8 MiB, resident on every GPU that loads the library
+static __device__ __align__(256) unsigned char g_decode_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static unsigned char *g_scratch_ptr[kMaxDevices] = {nullptr};   // device address of the array, per device
+
+// In host code `g_decode_scratch` is only a handle for the runtime; the address a kernel can
+// use has to be asked for, once per device, while that device is current.
+static int static_scratch_address(unsigned char **out)
+{
+    int dev = -1;
+    SP_CUDA(cudaGetDevice(&dev));
+    SP_REQUIRE(dev >= 0 && dev < kMaxDevices, SP_ERR_UNSUPPORTED,
+               "sp_pruned_decode_static: device ordinal %d not supported (max %d)", dev, kMaxDevices - 1);
+    if (g_scratch_ptr[dev] == nullptr) {
+        void *p = nullptr;
+        SP_CUDA(cudaGetSymbolAddress(&p, g_decode_scratch));
+        SP_REQUIRE(p != nullptr && aligned256(p), SP_ERR_CUDA,
+                   "sp_pruned_decode_static: the scratch array has no usable device address");
+        g_scratch_ptr[dev] = static_cast<unsigned char *>(p);
+    }
+    *out = g_scratch_ptr[dev];
+    return SP_OK;
+}
+
+}  // namespace sp
+
+extern "C" size_t sp_pruned_decode_static_max_bytes(void) { return sp::kStaticScratchBytes; }
+
+extern "C" int sp_pruned_decode_static(const void *q, const void *k_cache, const void *v_cache,
+                                       const sp_layout *lay, const int32_t *kept_idx, int k,
+                                       const void *tail_k, const void *tail_v,
+                                       const int32_t *tail_len, int tail_cap, int64_t max_keys,
+                                       int n_heads, int n_kv_heads, int head_dim, float scale,
+                                       void *out, float *lse, int dtype, void *stream)
+{
+    using namespace sp;
+    SP_REQUIRE(dtype == SP_F32 || dtype == SP_BF16, SP_ERR_INVALID_ARG, "sp_pruned_decode_static: unknown dtype %d", dtype);
+    if (int rc = check_layout(lay)) return rc;
+    SP_REQUIRE(head_dim == 64 || head_dim == 128, SP_ERR_UNSUPPORTED,
+               "sp_pruned_decode_static: head_dim %d (64 or 128 supported)", head_dim);
+    SP_REQUIRE(n_heads > 0 && n_kv_heads > 0 && n_heads % n_kv_heads == 0, SP_ERR_INVALID_ARG,
+               "sp_pruned_decode_static: n_heads %d must be a positive multiple of n_kv_heads %d", n_heads, n_kv_heads);
+    SP_REQUIRE(k >= 0 && k <= 4096, SP_ERR_INVALID_ARG, "sp_pruned_decode_static: k %d out of range [0, 4096]", k);
+    SP_REQUIRE(tail_cap >= 0 && max_keys >= 0, SP_ERR_INVALID_ARG, "sp_pruned_decode_static: negative tail_cap / max_keys");
+    SP_REQUIRE(lay->n_prompts <= 65535 && n_heads <= 65535, SP_ERR_UNSUPPORTED,
+               "sp_pruned_decode_static: more than 65535 prompts or heads");
+    if (lay->n_prompts == 0) return SP_OK;
+    SP_REQUIRE(q && out && k_cache && v_cache, SP_ERR_INVALID_ARG, "sp_pruned_decode_static: NULL tensor");
+    SP_REQUIRE(k == 0 || kept_idx, SP_ERR_INVALID_ARG, "sp_pruned_decode_static: kept_idx is NULL with k > 0");
+    SP_REQUIRE(tail_cap == 0 || (tail_k && tail_v && tail_len), SP_ERR_INVALID_ARG,
+               "sp_pruned_decode_static: tail pointers are NULL with tail_cap > 0");
+    SP_REQUIRE(aligned16(q) && aligned16(out) && aligned16(k_cache) && aligned16(v_cache) &&
+                   aligned16(tail_k) && aligned16(tail_v),
+               SP_ERR_INVALID_ARG, "sp_pruned_decode_static: data pointers must be 16-byte aligned");
+
+    if (max_keys == 0) max_keys = (int64_t)lay->max_pre_len + (int64_t)k * lay->max_path_len + tail_cap;
+    const int cap = decode_split_cap(lay->n_prompts, n_heads);
+    const int n_splits = (int)std::max<int64_t>(1, std::min<int64_t>(cap, (max_keys + 31) / 32));
+    const size_t cbytes = decode_counter_bytes(lay->n_prompts, n_heads);
+    const size_t pbytes = n_splits > 1
+        ? (size_t)lay->n_prompts * n_heads * n_splits * (head_dim + 2) * sizeof(float) : 0;
+    SP_REQUIRE(cbytes + pbytes <= kStaticScratchBytes, SP_ERR_WORKSPACE,
+               "sp_pruned_decode_static: this problem needs %zu bytes of split-KV scratch but the built-in "
+               "array holds %zu; use sp_pruned_decode with a caller workspace",
+               cbytes + pbytes, kStaticScratchBytes);
+
+    unsigned char *scratch = nullptr;
+    if (int rc = static_scratch_address(&scratch)) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array still holds the previous call's counters: they must start at zero
+    SP_CUDA(cudaMemsetAsync(scratch, 0, cbytes, st));
+
+    DecodeArgs a;
+    a.q = q; a.k_cache = k_cache; a.v_cache = v_cache; a.tail_k = tail_k; a.tail_v = tail_v;
+    a.ppo = lay->prompt_path_off; a.pre_start = lay->pre_start; a.pre_len = lay->pre_len;
+    a.path_start = lay->path_start; a.doc_len = lay->doc_len; a.qry_len = lay->qry_len;
+    a.kept_idx = kept_idx; a.tail_len = tail_len; a.out = out; a.lse = lse;
+    a.counters = reinterpret_cast<unsigned int *>(scratch);
+    a.partial = reinterpret_cast<float *>(scratch + cbytes);
+    a.k = k; a.tail_cap = tail_cap; a.n_heads = n_heads; a.n_kv_heads = n_kv_heads;
+    a.n_splits = n_splits; a.scale_log2e = scale * kLog2eD;
+
+    if (dtype == SP_BF16)
+        return head_dim == 128 ? launch_decode<__nv_bfloat16, 128>(a, lay->n_prompts, st)
+                               : launch_decode<__nv_bfloat16, 64>(a, lay->n_prompts, st);
+    return head_dim == 128 ? launch_decode<float, 128>(a, lay->n_prompts, st)
+                           : launch_decode<float, 64>(a, lay->n_prompts, st);
+}
