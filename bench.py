@@ -35,7 +35,7 @@ from workloads import (draw_decode_inputs, draw_lengths, draw_logits, draw_prior
 
 METRIC = "superposition prefill useful TFLOP/s over the whole hot-path step"
 UNIT = "TFLOP/s"
-PREFILL_LAUNCHES = 1           # kernels sp_superpose_prefill launches per call
+PREFILL_LAUNCHES = 2           # kernels sp_superpose_prefill launches per call (tile plan + attention)
 # dram__bytes_read.sum + dram__bytes_write.sum of one prefill launch, from the ncu capture
 # summarised under profiles/ (None until captured for the current kernel).
 NCU_PREFILL_TRAFFIC_BYTES = {}

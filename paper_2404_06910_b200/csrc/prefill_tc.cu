@@ -1,18 +1,446 @@
-// Placeholder until the tensor-core kernel lands: bf16 / head_dim 128 runs the SIMT kernel.
+// Fork-join prefill attention on the Blackwell tensor cores (bf16, head_dim 128).
+// Section 3.2: a row attends to its prompt's preamble and, causally, to its own path.
+//
+// Work unit: (128-row query tile of one segment, head).  Its keys are the preamble's rows
+// (all visible) followed by the segment's own rows up to the diagonal; key tiles that the
+// fork-join mask excludes are never loaded or multiplied.  Per key tile of up to 128 keys:
+//   S = Q K^T     tcgen05.mma, A and B from TMA-staged 128B-swizzled shared memory, fp32 in TMEM
+//   P = softmax   4 warps, one thread per query row (tcgen05.ld), online max / sum with lazy
+//                 rescaling, P rounded to bf16 and written over S in TMEM (tcgen05.st)
+//   O += P V      tcgen05.mma with A = P from TMEM, B = V from shared memory (MN-major)
+// Roles: warps 0-3 softmax + epilogue, warp 4 TMA producer, warp 5 MMA issuer / TMEM owner.
+// The grid is persistent; two blocks share an SM (256 TMEM columns each), so one block's
+// softmax overlaps the other's MMAs.  A small plan kernel turns the ragged layout into a
+// tile list.  Every mbarrier wait is bounded: on expiry the block records a timeout in the
+// workspace status word, unwinds, frees its TMEM and exits.
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace sp {
-int launch_prefill_simt(const void *q, const void *k, const void *v, const sp_layout *lay, int n_heads,
-                        int n_kv_heads, int head_dim, float scale, int rows, void *out, float *lse,
-                        int dtype, cudaStream_t st);
 
-size_t prefill_tc_workspace_bytes(int, int, int, int, int) { return 256; }
+using namespace ptx;
+
+constexpr int kBM = 128;              // query rows per tile
+constexpr int kBN = 128;              // keys per tile
+constexpr int kHD = 128;              // head_dim
+constexpr int kTcThreads = 192;
+constexpr int kTileBytes = kBM * kHD * 2;
+constexpr int kTmemCols = 256;        // S/P: [0,128)  O: [128,256)
+constexpr float kLog2eT = 1.4426950408889634f;
+constexpr float kLn2T = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.f;   // log2 units: rescale O only when the max grows by > 2^8
+
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+struct TcTile {                       // one 128-row query tile (shared by all heads)
+    int32_t q_row;                    // packed row of the tile's first query row
+    int32_t n_rows;                   // valid rows in the tile (1..128)
+    int32_t q_off;                    // offset of the first row inside its segment
+    int32_t own_row;                  // packed row of the segment's first row
+    int32_t pre_row, pre_len;         // fully visible prefix (the prompt's preamble), may be empty
+    int32_t pad0, pad1;
+};
+
+struct TcHeader {                     // start of the workspace
+    uint32_t status;
+    uint32_t n_tiles;
+};
+
+struct TcParams {
+    CUtensorMap mq, mk, mv;
+    const TcHeader *hdr;
+    const TcTile *tiles;
+    uint32_t *status;
+    __nv_bfloat16 *out;
+    float *lse;
+    int n_heads, kv_group;
+    int64_t total_tokens;
+    float scale_log2e;
+};
+
+// ---- plan: ragged layout -> tile list ---------------------------------------------------
+struct PlanArgs {
+    const int32_t *ppo, *pre_start, *pre_len, *path_start, *doc_len, *qry_len;
+    int n_prompts, n_paths, rows_mode;
+    TcHeader *hdr;
+    TcTile *tiles;
+};
+
+__global__ void __launch_bounds__(1024) prefill_plan_kernel(const PlanArgs a)
+{
+    __shared__ int warp_tot[32];
+    __shared__ int running;
+    if (threadIdx.x == 0) running = 0;
+    __syncthreads();
+    const int n_seq = a.n_prompts + a.n_paths;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int base = 0; base < n_seq; base += 1024) {
+        const int s = base + threadIdx.x;
+        int first = 0, rows = 0, own_row = 0, pre_row = 0, pre_n = 0;
+        if (s < a.n_prompts) {
+            if (a.rows_mode == SP_ROWS_ALL) { rows = a.pre_len[s]; own_row = a.pre_start[s]; }
+        } else if (s < n_seq) {
+            const int i = s - a.n_prompts;
+            int lo = 0, hi = a.n_prompts - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (a.ppo[mid] <= i) lo = mid; else hi = mid - 1;
+            }
+            pre_row = a.pre_start[lo]; pre_n = a.pre_len[lo];
+            own_row = a.path_start[i];
+            first = a.rows_mode == SP_ROWS_QUERY_ONLY ? a.doc_len[i] : 0;
+            rows = a.doc_len[i] + a.qry_len[i] - first;
+        }
+        const int nt = (rows + kBM - 1) / kBM;
+        int incl = nt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        int before = running;
+        for (int w = 0; w < warp; ++w) before += warp_tot[w];
+        int off = before + incl - nt;
+        for (int t = 0; t < nt; ++t) {
+            TcTile tl;
+            tl.q_off = first + t * kBM;
+            tl.q_row = own_row + tl.q_off;
+            tl.n_rows = min(kBM, rows - t * kBM);
+            tl.own_row = own_row;
+            tl.pre_row = pre_row; tl.pre_len = pre_n; tl.pad0 = 0; tl.pad1 = 0;
+            a.tiles[off + t] = tl;
+        }
+        __syncthreads();
+        if (threadIdx.x == 1023) running = before + incl;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) a.hdr->n_tiles = (uint32_t)running;
+}
+
+// Key tile j of a query tile: preamble tiles first, then the segment's own rows up to the
+// tile's last valid query row.
+struct KvTile {
+    int row0;        // packed row of the first key
+    int n_valid;     // keys that exist (1..128)
+    int k_off;       // own-segment offset of the first key; -1 for preamble tiles (no causal limit)
+};
+__device__ __forceinline__ int n_kv_tiles(const TcTile &t)
+{
+    return (t.pre_len + kBN - 1) / kBN + (t.q_off + t.n_rows + kBN - 1) / kBN;
+}
+__device__ __forceinline__ KvTile kv_tile(const TcTile &t, int j)
+{
+    const int n_pre = (t.pre_len + kBN - 1) / kBN;
+    KvTile k;
+    if (j < n_pre) {
+        k.row0 = t.pre_row + j * kBN; k.n_valid = min(kBN, t.pre_len - j * kBN); k.k_off = -1;
+    } else {
+        const int o = (j - n_pre) * kBN;
+        k.row0 = t.own_row + o; k.n_valid = min(kBN, t.q_off + t.n_rows - o); k.k_off = o;
+    }
+    return k;
+}
+
+enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_K_EMPTY, BAR_V_FULL, BAR_V_EMPTY, BAR_S_FULL, BAR_P_FULL,
+       BAR_O_DONE, BAR_COUNT };
+
+__global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_constant__ TcParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    unsigned char *sQ = smem, *sK = smem + kTileBytes, *sV = smem + 2 * kTileBytes;
+    __shared__ uint64_t bars[BAR_COUNT];
+    __shared__ uint32_t tmem_base_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < BAR_COUNT; ++i) mbar_init(&bars[i], i == BAR_P_FULL ? 128 : 1);
+        fence_mbar_init();
+        prefetch_tmap(&p.mq); prefetch_tmap(&p.mk); prefetch_tmap(&p.mv);
+    }
+    if (warp == 5) { tmem_alloc(&tmem_base_s, kTmemCols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tb = tmem_base_s;
+    const uint32_t n_items = p.hdr->n_tiles * (uint32_t)p.n_heads;
+    bool ok = true;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t qe = 0, ke = 0, ve = 0;
+            uint32_t nq = 0, nk = 0, nv = 0;          // loads issued per "full" barrier
+            for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+                const TcTile t = p.tiles[it / p.n_heads];
+                const int h = it % p.n_heads, hk = h / p.kv_group;
+                if (!(ok = mbar_wait(&bars[BAR_Q_EMPTY], qe ^ 1))) break;
+                qe ^= 1;
+                mbar_expect_tx(&bars[BAR_Q_FULL], kTileBytes);
+                tma_load_2d(sQ, &p.mq, h * kHD, t.q_row, &bars[BAR_Q_FULL]);
+                tma_load_2d(sQ + kTileBytes / 2, &p.mq, h * kHD + 64, t.q_row, &bars[BAR_Q_FULL]);
+                ++nq;
+                const int n_kv = n_kv_tiles(t);
+                for (int j = 0; j < n_kv; ++j) {
+                    const KvTile kt = kv_tile(t, j);
+                    if (!(ok = mbar_wait(&bars[BAR_K_EMPTY], ke ^ 1))) break;
+                    ke ^= 1;
+                    mbar_expect_tx(&bars[BAR_K_FULL], kTileBytes);
+                    tma_load_2d(sK, &p.mk, hk * kHD, kt.row0, &bars[BAR_K_FULL]);
+                    tma_load_2d(sK + kTileBytes / 2, &p.mk, hk * kHD + 64, kt.row0, &bars[BAR_K_FULL]);
+                    ++nk;
+                    if (!(ok = mbar_wait(&bars[BAR_V_EMPTY], ve ^ 1))) break;
+                    ve ^= 1;
+                    mbar_expect_tx(&bars[BAR_V_FULL], kTileBytes);
+                    tma_load_2d(sV, &p.mv, hk * kHD, kt.row0, &bars[BAR_V_FULL]);
+                    tma_load_2d(sV + kTileBytes / 2, &p.mv, hk * kHD + 64, kt.row0, &bars[BAR_V_FULL]);
+                    ++nv;
+                }
+            }
+            if (!ok) {
+                // a wait ran out: before the block may exit, its own copies in flight must
+                // have landed (bounded waits on the phase of the last load of each buffer)
+                if (nq) mbar_wait(&bars[BAR_Q_FULL], (nq - 1) & 1);
+                if (nk) mbar_wait(&bars[BAR_K_FULL], (nk - 1) & 1);
+                if (nv) mbar_wait(&bars[BAR_V_FULL], (nv - 1) & 1);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t qf = 0, kf = 0, vf = 0, pf = 0;
+            const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
+            for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+                const TcTile t = p.tiles[it / p.n_heads];
+                if (!(ok = mbar_wait(&bars[BAR_Q_FULL], qf))) break;
+                qf ^= 1;
+                const int n_kv = n_kv_tiles(t);
+                for (int j = 0; j < n_kv; ++j) {
+                    const KvTile kt = kv_tile(t, j);
+                    const int n_mma = (kt.n_valid + 15) & ~15;
+                    if (!(ok = mbar_wait(&bars[BAR_K_FULL], kf))) break;
+                    kf ^= 1;
+                    tc_fence_after();
+                    const uint32_t id_s = idesc_bf16(kBM, n_mma, 0, 0);
+#pragma unroll
+                    for (int kk = 0; kk < kHD / 16; ++kk) {          // contraction over head_dim
+                        const uint32_t off = (kk >> 2) * (kTileBytes / 2) + (kk & 3) * 32;
+                        umma_ss(tb, smem_desc_sw128(aQ + off, 16, 1024), smem_desc_sw128(aK + off, 16, 1024), id_s, kk > 0);
+                    }
+                    umma_commit(&bars[BAR_S_FULL]);
+                    umma_commit(&bars[BAR_K_EMPTY]);
+                    if (j == n_kv - 1) umma_commit(&bars[BAR_Q_EMPTY]);
+                    if (!(ok = mbar_wait(&bars[BAR_P_FULL], pf))) break;
+                    pf ^= 1;
+                    if (!(ok = mbar_wait(&bars[BAR_V_FULL], vf))) break;
+                    vf ^= 1;
+                    tc_fence_after();
+                    const uint32_t id_o = idesc_bf16(kBM, kHD, 0, 1);
+                    for (int kk = 0; kk < n_mma / 16; ++kk)          // contraction over keys
+                        umma_ts(tb + 128, tb + kk * 8, smem_desc_sw128(aV + kk * 2048, kTileBytes / 2, 1024), id_o,
+                                (j > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(&bars[BAR_V_EMPTY]);
+                    if (j == n_kv - 1) umma_commit(&bars[BAR_O_DONE]);
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ softmax + epilogue
+        uint32_t sf = 0, od = 0;
+        const int row = warp * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        const float sc = p.scale_log2e;
+        for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+            const TcTile t = p.tiles[it / p.n_heads];
+            const int h = it % p.n_heads;
+            const int n_kv = n_kv_tiles(t);
+            float m_ref = -INFINITY, l = 0.f;
+            for (int j = 0; j < n_kv; ++j) {
+                const KvTile kt = kv_tile(t, j);
+                const int n_mma = (kt.n_valid + 15) & ~15;
+                const int n_chunks = (n_mma + 31) >> 5;
+                // visible keys of this row / of the warp's last row in this tile
+                const int lim = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + row - kt.k_off + 1);
+                const int wlim = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + warp * 32 + 31 - kt.k_off + 1);
+                if (!(ok = mbar_wait(&bars[BAR_S_FULL], sf))) break;
+                sf ^= 1;
+                tc_fence_after();
+
+                float tmax = -INFINITY;
+                for (int c = 0; c < n_chunks && c * 32 < wlim; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tb + lane_addr + c * 32, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        tmax = fmaxf(tmax, (c * 32 + i < lim) ? __uint_as_float(r[i]) : -INFINITY);
+                }
+                const float m_tile = tmax * sc;
+                float alpha = 1.f;
+                bool grow = false;
+                if (j == 0) {
+                    m_ref = m_tile;
+                } else if (m_tile > m_ref + kRescaleThreshold) {
+                    alpha = ex2(m_ref - m_tile);
+                    m_ref = m_tile;
+                    grow = true;
+                }
+                if (__any_sync(0xffffffffu, grow)) {     // rare: bring O and l to the new reference
+                    l *= alpha;
+                    for (int c = 0; c < kHD / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(tb + lane_addr + 128 + c * 32, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                        tmem_st32(tb + lane_addr + 128 + c * 32, r);
+                    }
+                }
+                for (int c = 0; c < n_chunks; ++c) {
+                    uint32_t pk[16];
+                    if (c * 32 < wlim) {
+                        uint32_t r[32];
+                        tmem_ld32(tb + lane_addr + c * 32, r);
+                        tmem_ld_wait();
+                        float rs = 0.f;
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) {
+                            const float x0 = fmaf(__uint_as_float(r[i]), sc, -m_ref);
+                            const float x1 = fmaf(__uint_as_float(r[i + 1]), sc, -m_ref);
+                            const float p0 = (c * 32 + i < lim) ? ex2(x0) : 0.f;
+                            const float p1 = (c * 32 + i + 1 < lim) ? ex2(x1) : 0.f;
+                            rs += p0 + p1;
+                            pk[i >> 1] = pack_bf16x2(p0, p1);
+                        }
+                        l += rs;
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) pk[i] = 0u;
+                    }
+                    tmem_st16(tb + lane_addr + c * 16, pk);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(&bars[BAR_P_FULL]);
+            }
+            if (!ok) break;
+            if (!(ok = mbar_wait(&bars[BAR_O_DONE], od))) break;
+            od ^= 1;
+            tc_fence_after();
+            const float inv = 1.f / l;
+            const bool live = row < t.n_rows;
+            __nv_bfloat16 *dst = p.out + ((int64_t)(t.q_row + row) * p.n_heads + h) * kHD;
+            for (int c = 0; c < kHD / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tb + lane_addr + 128 + c * 32, r);
+                tmem_ld_wait();
+                if (live) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
+                        w.y = pack_bf16x2(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+                        w.z = pack_bf16x2(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
+                        w.w = pack_bf16x2(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(dst + c * 32 + i) = w;
+                    }
+                }
+            }
+            if (live && p.lse) p.lse[(int64_t)h * p.total_tokens + t.q_row + row] = (m_ref + log2f(l)) * kLn2T;
+            tc_fence_before();
+        }
+    }
+
+    if (!ok && lane == 0) atomicExch(p.status, (uint32_t)STATUS_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) tmem_dealloc(tb, kTmemCols);
+}
+
+// ---- host side ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static int encode_rows_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int64_t rows, int64_t cols)
+{
+    // [rows, cols] bf16 row-major; box = 128 rows x 64 columns (128 bytes), 128-byte swizzle
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kBM};
+    cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    SP_REQUIRE(r == CUDA_SUCCESS, SP_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return SP_OK;
+}
+
+static int64_t max_tiles(int n_prompts, int n_paths, int max_pre_len, int max_path_len)
+{
+    return (int64_t)n_prompts * ((max_pre_len + kBM - 1) / kBM) + (int64_t)n_paths * ((max_path_len + kBM - 1) / kBM);
+}
+
+size_t prefill_tc_workspace_bytes(int n_prompts, int n_paths, int max_pre_len, int max_path_len, int)
+{
+    if (n_prompts < 0 || n_paths < 0 || max_pre_len < 0 || max_path_len < 0) return 256;
+    return 256 + round_up((size_t)max_tiles(n_prompts, n_paths, max_pre_len, max_path_len) * sizeof(TcTile), 256);
+}
 
 int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layout *lay, int n_heads,
                       int n_kv_heads, float scale, int rows, void *out, float *lse, void *ws,
                       size_t, cudaStream_t st)
 {
+    static EncodeTiledFn enc = nullptr;
+    if (!enc) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        SP_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+        SP_REQUIRE(fn != nullptr && qres == cudaDriverEntryPointSuccess, SP_ERR_CUDA,
+                   "cuTensorMapEncodeTiled is not available from this driver");
+        enc = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    SP_REQUIRE(((int64_t)n_heads * kHD * 2) % 16 == 0, SP_ERR_INVALID_ARG, "row stride must be a multiple of 16 bytes");
+
+    TcParams p;
+    if (int rc = encode_rows_map(enc, &p.mq, q, lay->total_tokens, (int64_t)n_heads * kHD)) return rc;
+    if (int rc = encode_rows_map(enc, &p.mk, k, lay->total_tokens, (int64_t)n_kv_heads * kHD)) return rc;
+    if (int rc = encode_rows_map(enc, &p.mv, v, lay->total_tokens, (int64_t)n_kv_heads * kHD)) return rc;
+
+    TcHeader *hdr = static_cast<TcHeader *>(ws);
+    TcTile *tiles = reinterpret_cast<TcTile *>(static_cast<char *>(ws) + 256);
     SP_CUDA(cudaMemsetAsync(ws, 0, 256, st));
-    return launch_prefill_simt(q, k, v, lay, n_heads, n_kv_heads, 128, scale, rows, out, lse, SP_BF16, st);
+
+    PlanArgs pa;
+    pa.ppo = lay->prompt_path_off; pa.pre_start = lay->pre_start; pa.pre_len = lay->pre_len;
+    pa.path_start = lay->path_start; pa.doc_len = lay->doc_len; pa.qry_len = lay->qry_len;
+    pa.n_prompts = lay->n_prompts; pa.n_paths = lay->n_paths; pa.rows_mode = rows;
+    pa.hdr = hdr; pa.tiles = tiles;
+    prefill_plan_kernel<<<1, 1024, 0, st>>>(pa);
+    SP_CUDA(cudaGetLastError());
+
+    p.hdr = hdr; p.tiles = tiles; p.status = &hdr->status;
+    p.out = static_cast<__nv_bfloat16 *>(out); p.lse = lse;
+    p.n_heads = n_heads; p.kv_group = n_heads / n_kv_heads;
+    p.total_tokens = lay->total_tokens; p.scale_log2e = scale * kLog2eT;
+
+    const int64_t items = max_tiles(lay->n_prompts, lay->n_paths, lay->max_pre_len, lay->max_path_len) * n_heads;
+    if (items == 0) return SP_OK;
+    const int grid = (int)std::min<int64_t>(items, 2 * kNumSMs);
+    const int smem = 3 * kTileBytes + 1024;
+    SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    prefill_tc_kernel<<<grid, kTcThreads, smem, st>>>(p);
+    SP_CUDA(cudaGetLastError());
+    return SP_OK;
 }
+
 }  // namespace sp
