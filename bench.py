@@ -110,14 +110,14 @@ class ClockSampler:
 class HotPath:
     """Device buffers and the launch sequence of one step, through the C-ABI binding."""
 
-    def __init__(self, cfg, seed, sp, device):
+    def __init__(self, cfg, seed, sp, device, n_prompts=None, decode_steps=None):
         self.cfg, self.sp = cfg, sp
         t0 = time.time()
-        self.lay = lay = draw_lengths(cfg, seed=seed)
+        self.lay = lay = draw_lengths(cfg, seed=seed, n_prompts=n_prompts)
         B, H, Hkv, D = lay.n_prompts, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim
         self.B, self.H, self.Hkv, self.D = B, H, Hkv, D
         self.tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
-        self.steps_dec = cfg.decode_steps
+        self.steps_dec = cfg.decode_steps if decode_steps is None else decode_steps
         # host inputs (pinned: they are also the source of the end-to-end copies)
         self.h_q, self.h_k, self.h_v = draw_qkv(cfg, lay, seed=seed, pin=True)
         self.h_logits = draw_logits(cfg, lay, seed=seed, pin=True)
@@ -232,7 +232,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
     cfg = get_config(args.workload)
-    hp = HotPath(cfg, cfg.seed + 1000 * rank, sp, device)
+    hp = HotPath(cfg, cfg.seed + 1000 * rank, sp, device, args.prompts, args.decode_steps)
     peaks = load_peaks()
     l2_bytes = torch.cuda.get_device_properties(device).L2_cache_size
     flush = None
@@ -275,17 +275,20 @@ def run_ours(args):
     ms_per_step = total_ms / args.steps
 
     # end to end: pinned host -> device copies of every input, the pass, device -> host results
-    e2e_steps = max(1, min(args.steps, 3))
-    hp.h2d(); hp.step(); hp.d2h(); sync()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(e2e_steps):
-        bi = hp.h2d()
-        hp.step()
-        bo = hp.d2h()
-    e1.record()
-    sync()
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 3))
+    bi = bo = 0
+    e2e_ms = float("nan")
+    if e2e_steps:
+        hp.h2d(); hp.step(); hp.d2h(); sync()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e2e_steps):
+            bi = hp.h2d()
+            hp.step()
+            bo = hp.d2h()
+        e1.record()
+        sync()
+        e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
     t = torch.tensor([ms_per_step, e2e_ms], dtype=torch.float64, device=device)
     if dist is not None:
@@ -328,8 +331,9 @@ def run_ours(args):
                          "algorithmic_bytes": hp.bytes_prefill, "useful_tflops": pre_tf,
                          "frac_bf16_sustained": pre_tf / peaks["bf16_tflops_sustained"]},
             "kernels": kernels,
-            "e2e": {"value": world * tf(hp.flop_prefill, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
-                    "steps": e2e_steps, "h2d_bytes_per_step": bi, "d2h_bytes_per_step": bo},
+            "e2e": None if not e2e_steps else {
+                "value": world * tf(hp.flop_prefill, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
+                "steps": e2e_steps, "h2d_bytes_per_step": bi, "d2h_bytes_per_step": bo},
             "gpu_launches": hp.launches * args.steps,
             "clocks": clocks,
             "input_generation_s": hp.gen_s,
@@ -420,6 +424,9 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling aid)")
+    ap.add_argument("--prompts", type=int, default=None, help="override the prompts per GPU (profiling aid)")
+    ap.add_argument("--decode-steps", type=int, default=None, help="override the decode steps (profiling aid)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

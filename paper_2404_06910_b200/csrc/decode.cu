@@ -12,7 +12,7 @@
 namespace sp {
 
 constexpr int kDecThreads = 128;
-constexpr int kDecUnroll = 4;        // keys in flight per key group
+constexpr int kDecUnroll = 8;        // keys in flight per key group
 constexpr int kDecMaxSplits = 64;
 constexpr float kLog2eD = 1.4426950408889634f;
 constexpr float kLn2D = 0.6931471805599453f;
@@ -48,8 +48,29 @@ static int decode_split_cap(int n_prompts, int n_heads)
     return (int)std::min<int64_t>(kDecMaxSplits, std::max<int64_t>(1, want));
 }
 
+// 16 bytes of a key / value row, kept raw until the arithmetic needs them.
+__device__ __forceinline__ uint4 ld_stream16(const void *p)
+{
+    uint4 w;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w) : "l"(p));
+    return w;
+}
+template <typename T> struct Raw16;
+template <> struct Raw16<__nv_bfloat16> {
+    __device__ __forceinline__ static void unpack(const uint4 &w, float (&f)[8]) {
+        f[0] = bf16_lo(w.x); f[1] = bf16_hi(w.x); f[2] = bf16_lo(w.y); f[3] = bf16_hi(w.y);
+        f[4] = bf16_lo(w.z); f[5] = bf16_hi(w.z); f[6] = bf16_lo(w.w); f[7] = bf16_hi(w.w);
+    }
+};
+template <> struct Raw16<float> {
+    __device__ __forceinline__ static void unpack(const uint4 &w, float (&f)[4]) {
+        f[0] = __uint_as_float(w.x); f[1] = __uint_as_float(w.y); f[2] = __uint_as_float(w.z); f[3] = __uint_as_float(w.w);
+    }
+};
+
 template <typename T, int D>
-__global__ void __launch_bounds__(kDecThreads)
+__global__ void __launch_bounds__(kDecThreads, 5)
 decode_kernel(const __grid_constant__ DecodeArgs a)
 {
     constexpr int N = Vec<T>::N;            // elements per 16-byte load
@@ -70,27 +91,34 @@ decode_kernel(const __grid_constant__ DecodeArgs a)
     const int hk = h / (a.n_heads / a.n_kv_heads);
     const int64_t row_elems = (int64_t)a.n_kv_heads * D;
 
-    if (threadIdx.x == 0) {
+    // segments: 0 = preamble, 1..k = kept paths, k+1 = tail; lengths land in seg_lo[s+1]
+    for (int sgm = threadIdx.x; sgm < n_seg; sgm += kDecThreads) {
         const T *kc = static_cast<const T *>(a.k_cache) + (int64_t)hk * D;
         const T *vc = static_cast<const T *>(a.v_cache) + (int64_t)hk * D;
+        int len = 0;
+        int64_t row = 0;
+        if (sgm == 0) {
+            row = a.pre_start[b]; len = a.pre_len[b];
+        } else if (sgm <= a.k) {
+            const int i = a.kept_idx[(int64_t)b * a.k + sgm - 1];
+            if (i >= a.ppo[b] && i < a.ppo[b + 1]) { row = a.path_start[i]; len = a.doc_len[i] + a.qry_len[i]; }
+        } else {
+            len = (a.tail_cap > 0 && a.tail_len) ? min(max(a.tail_len[b], 0), a.tail_cap) : 0;
+            if (len) {
+                kc = static_cast<const T *>(a.tail_k) + (int64_t)hk * D;
+                vc = static_cast<const T *>(a.tail_v) + (int64_t)hk * D;
+                row = (int64_t)b * a.tail_cap;
+            }
+        }
+        seg_k[sgm] = kc + row * row_elems;
+        seg_v[sgm] = vc + row * row_elems;
+        seg_lo[sgm + 1] = len;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
         int cum = 0;
         seg_lo[0] = 0;
-        seg_k[0] = kc + (int64_t)a.pre_start[b] * row_elems;
-        seg_v[0] = vc + (int64_t)a.pre_start[b] * row_elems;
-        cum += a.pre_len[b];
-        for (int j = 0; j < a.k; ++j) {
-            const int i = a.kept_idx[(int64_t)b * a.k + j];
-            const bool ok = i >= a.ppo[b] && i < a.ppo[b + 1];
-            seg_lo[j + 1] = cum;
-            seg_k[j + 1] = ok ? kc + (int64_t)a.path_start[i] * row_elems : kc;
-            seg_v[j + 1] = ok ? vc + (int64_t)a.path_start[i] * row_elems : vc;
-            cum += ok ? a.doc_len[i] + a.qry_len[i] : 0;
-        }
-        seg_lo[a.k + 1] = cum;
-        const int tl = (a.tail_cap > 0 && a.tail_len) ? min(max(a.tail_len[b], 0), a.tail_cap) : 0;
-        seg_k[a.k + 1] = tl ? static_cast<const T *>(a.tail_k) + ((int64_t)b * a.tail_cap) * row_elems + (int64_t)hk * D : kc;
-        seg_v[a.k + 1] = tl ? static_cast<const T *>(a.tail_v) + ((int64_t)b * a.tail_cap) * row_elems + (int64_t)hk * D : vc;
-        seg_lo[n_seg] = cum + tl;
+        for (int sgm = 0; sgm < n_seg; ++sgm) { cum += seg_lo[sgm + 1]; seg_lo[sgm + 1] = cum; }
     }
     __syncthreads();
 
@@ -110,17 +138,17 @@ decode_kernel(const __grid_constant__ DecodeArgs a)
 
     int seg = 0;
     for (int base = lo; base < hi; base += G * kDecUnroll) {   // trip count is block-uniform
-        float kf[kDecUnroll][N], vf[kDecUnroll][N];
+        uint4 kr[kDecUnroll], vr[kDecUnroll];
         bool live[kDecUnroll];
 #pragma unroll
-        for (int u = 0; u < kDecUnroll; ++u) {
+        for (int u = 0; u < kDecUnroll; ++u) {                  // all loads of the batch first
             const int j = base + g + u * G;
             live[u] = j < hi;
             if (live[u]) {
-                while (j >= seg_lo[seg + 1]) ++seg;        // keys ascend: segments only advance
+                while (j >= seg_lo[seg + 1]) ++seg;             // keys ascend: segments only advance
                 const int64_t off = (int64_t)(j - seg_lo[seg]) * row_elems + sub * N;
-                Vec<T>::load(seg_k[seg] + off, kf[u]);
-                Vec<T>::load(seg_v[seg] + off, vf[u]);
+                kr[u] = ld_stream16(seg_k[seg] + off);
+                vr[u] = ld_stream16(seg_v[seg] + off);
             }
         }
         float s[kDecUnroll], cm = -INFINITY;
@@ -128,8 +156,10 @@ decode_kernel(const __grid_constant__ DecodeArgs a)
         for (int u = 0; u < kDecUnroll; ++u) {
             float d = 0.f;
             if (live[u]) {
+                float kf[N];
+                Raw16<T>::unpack(kr[u], kf);
 #pragma unroll
-                for (int e = 0; e < N; ++e) d = fmaf(qf[e], kf[u][e], d);
+                for (int e = 0; e < N; ++e) d = fmaf(qf[e], kf[e], d);
             }
 #pragma unroll
             for (int o = LPK / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
@@ -148,8 +178,10 @@ decode_kernel(const __grid_constant__ DecodeArgs a)
             if (live[u]) {
                 const float p = ex2f(s[u] - m);
                 l += p;
+                float vf[N];
+                Raw16<T>::unpack(vr[u], vf);
 #pragma unroll
-                for (int e = 0; e < N; ++e) acc[e] = fmaf(p, vf[u][e], acc[e]);
+                for (int e = 0; e < N; ++e) acc[e] = fmaf(p, vf[e], acc[e]);
             }
         }
     }
