@@ -167,6 +167,7 @@ class HotPath:
         # kernels launched per step (ours): rope x2, prefill, row_logp + path_sum, top-k,
         # per decode step rope x2 + decode
         self.launches = 2 + PREFILL_LAUNCHES + 2 + 1 + self.steps_dec * 3
+        self.decode_graph = None
 
     def decode_bytes(self):
         kept = self.kept.cpu().numpy()
@@ -206,13 +207,37 @@ class HotPath:
         mark()
         sp.sp_prune_topk(self.scores, self.dl.prompt_path_off, cfg.top_k, self.kept, self.post)
         mark()
+        if self.decode_graph is not None:
+            self.decode_graph.replay()
+        else:
+            self.decode_loop()
+        mark()
+
+    def decode_loop(self):
+        sp, cfg = self.sp, self.cfg
+        H, Hkv, D, B = self.H, self.Hkv, self.D, self.B
         ld = self.steps_dec * Hkv * D
         for t in range(self.steps_dec):
             sp.sp_rope_apply(self.dq[t], self.tpos[t], H, D, base=cfg.rope_base)
             sp.sp_rope_apply(self.tk[:, t], self.tpos[t], Hkv, D, n_tokens=B, ld_token=ld, base=cfg.rope_base)
             sp.sp_pruned_decode(self.dq[t], self.k, self.v, self.dl, self.kept, cfg.top_k, self.tk, self.tv,
                                 self.tail_len[t], self.steps_dec, self.scale, self.dec_out[t], None, self.ws_dec)
-        mark()
+
+    def capture_decode_graph(self):
+        """The decode loop is launch-bound (3 small launches per token): replay it from a CUDA
+        graph.  kept_idx is read on the device, so the captured graph stays valid when the
+        kept set changes."""
+        self.kept.fill_(-1)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            self.decode_loop()                      # warm-up outside capture (first-call set-up)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            self.decode_loop()
+        self.decode_graph = g
 
 
 STAGES = ("rope", "prefill", "path_scores", "topk", "decode")
@@ -233,6 +258,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=device)
     cfg = get_config(args.workload)
     hp = HotPath(cfg, cfg.seed + 1000 * rank, sp, device, args.prompts, args.decode_steps)
+    if not args.no_graph:
+        hp.capture_decode_graph()
     peaks = load_peaks()
     l2_bytes = torch.cuda.get_device_properties(device).L2_cache_size
     flush = None
@@ -313,7 +340,7 @@ def run_ours(args):
             "topk": {"ms": ms["topk"]},
             "decode": {"ms": ms["decode"], "steps": hp.steps_dec, "gbs": gb(hp.bytes_decode, ms["decode"]),
                        "frac_hbm": gb(hp.bytes_decode, ms["decode"]) / peaks["hbm_gbs"],
-                       "includes": "2 rope launches + 1 decode launch per token"},
+                       "includes": "2 rope launches + 1 decode launch per token" + ("" if args.no_graph else ", replayed from a CUDA graph")},
         }
         line = {
             "metric": METRIC, "value": world * tf(hp.flop_prefill, ms_per_step), "unit": UNIT,
@@ -339,7 +366,7 @@ def run_ours(args):
             "input_generation_s": hp.gen_s,
         }
         if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(cfg, steps=1, warmup=0, budget_s=25.0)[0]
+            line["cpu_baseline"] = cpu_baseline(cfg, steps=1, warmup=0, budget_s=15.0)[0]
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()
@@ -347,48 +374,50 @@ def run_ours(args):
 
 
 # ---------------------------------------------------------------------------------------
-def oracle_sample_pass(cfg, n_paths):
-    """Returns a closure running the whole hot path in the CPU oracle on the first n_paths
-    paths of prompt 0 of the workload, and the useful prefill FLOPs of that sample."""
+def oracle_sample_pass(cfg, n_prompts):
+    """Returns a closure that runs the whole hot path in the CPU oracle on the first n_prompts
+    prompts of the workload, and the useful prefill FLOPs of that sample."""
     import oracle
-    from workloads import build_layout
     from workloads.tensors import to_f32_numpy
-    full = draw_lengths(cfg)
-    n_paths = min(n_paths, int(full.prompt_path_off[1]))
-    lay = build_layout([int(full.pre_len[0])], [full.doc_len[:n_paths]], [full.qry_len[:n_paths]])
+    lay = draw_lengths(cfg, n_prompts=n_prompts)
+    B = lay.n_prompts
     q, k, v = (to_f32_numpy(t) for t in draw_qkv(cfg, lay))
     logits = to_f32_numpy(draw_logits(cfg, lay))
     tgt = draw_targets(cfg, lay)
     prior, weight = draw_prior_weight(cfg, lay)
     steps = cfg.decode_steps
-    dq, tk, tv = (to_f32_numpy(t) for t in draw_decode_inputs(cfg, 1, steps))
+    dq, tk, tv = (to_f32_numpy(t) for t in draw_decode_inputs(cfg, B, steps))
     scheme = "equilibrium" if cfg.positions == "equilibrium" else "left"
     scale = 1.0 / math.sqrt(cfg.head_dim)
-    kk = min(cfg.top_k, n_paths)
 
     def run():
-        pos, _, nxt = oracle.positions(int(lay.pre_len[0]), lay.doc_len, int(lay.qry_len[0]), scheme=scheme)
-        pos = pos.astype(np.float32)
+        pos, nxt = positions_all(lay, lambda P, L, Q: oracle.positions(P, L, Q, scheme=scheme))
         qr = oracle.rope(q, pos, base=cfg.rope_base)
         kr = oracle.rope(k, pos, base=cfg.rope_base)
         oracle.prefill(qr, kr, v, lay, scale)
         s, _ = oracle.path_scores(logits, tgt, lay.query_row_offsets(), prior, weight)
-        kept, _ = oracle.prune_topk(s, lay.prompt_path_off, kk)
+        kept, _ = oracle.prune_topk(s, lay.prompt_path_off, cfg.top_k)
         tkr = tk.copy()
         for t in range(steps):
-            tp = np.array([nxt + t], np.float32)
+            tp = (nxt + t).astype(np.float32)
             qt = oracle.rope(dq[t], tp, base=cfg.rope_base)
             tkr[:, t] = oracle.rope(np.ascontiguousarray(tkr[:, t]), tp, base=cfg.rope_base)
-            oracle.pruned_decode(qt, kr, v, lay, kept, tkr, tv, np.array([t + 1], np.int32), scale)
+            oracle.pruned_decode(qt, kr, v, lay, kept, tkr, tv, np.full(B, t + 1, np.int32), scale)
 
     flop = 4.0 * cfg.head_dim * cfg.n_heads * lay.allowed_pairs()
-    return run, flop, n_paths
+    return run, flop, B
 
 
 def cpu_baseline(cfg, steps, warmup, budget_s):
+    """Times the oracle, as it stands, on a bounded sample: whole prompts of the workload,
+    as many as fit the time budget (calibrated on one prompt)."""
     import oracle
-    n_paths = int(max(1, min(cfg.n_docs, (budget_s / max(1, steps + warmup)) // 0.4)))
-    run, flop, n_paths = oracle_sample_pass(cfg, n_paths)
+    run1, _, _ = oracle_sample_pass(cfg, 1)
+    t0 = time.perf_counter()
+    run1()
+    t1 = max(time.perf_counter() - t0, 1e-3)
+    n = int(max(1, min(cfg.n_prompts, budget_s / max(1, steps + warmup) / t1)))
+    run, flop, n = oracle_sample_pass(cfg, n)
     for _ in range(warmup):
         run()
     t0 = time.perf_counter()
@@ -396,8 +425,8 @@ def cpu_baseline(cfg, steps, warmup, budget_s):
         run()
     dt = (time.perf_counter() - t0) / steps
     return ({"value": flop / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-             "sample": f"whole hot path on prompt 0 restricted to its first {n_paths} paths "
-                       f"({cfg.name}, all heads, {cfg.decode_steps} decode steps)",
+             "sample": f"whole hot path (rope, prefill, scores, top-k, {cfg.decode_steps} decode steps) on the "
+                       f"first {n} of {cfg.n_prompts} prompts of {cfg.name}, all heads",
              "ms_per_sample": dt * 1e3}, dt)
 
 
@@ -424,6 +453,7 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch the decode loop eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling aid)")
     ap.add_argument("--prompts", type=int, default=None, help="override the prompts per GPU (profiling aid)")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the decode steps (profiling aid)")

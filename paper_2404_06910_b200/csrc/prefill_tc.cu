@@ -3,14 +3,16 @@
 //
 // Work unit: (128-row query tile of one segment, head).  Its keys are the preamble's rows
 // (all visible) followed by the segment's own rows up to the diagonal; key tiles that the
-// fork-join mask excludes are never loaded or multiplied.  Per key tile of up to 128 keys:
+// fork-join mask excludes are never loaded or multiplied.  Per key tile of up to 64 keys:
 //   S = Q K^T     tcgen05.mma, A and B from TMA-staged 128B-swizzled shared memory, fp32 in TMEM
-//   P = softmax   4 warps, one thread per query row (tcgen05.ld), online max / sum with lazy
-//                 rescaling, P rounded to bf16 and written over S in TMEM (tcgen05.st)
+//   P = softmax   4 warps, one thread per query row (tcgen05.ld, the row stays in registers),
+//                 online max / sum with lazy rescaling, P rounded to bf16 and written over S
+//                 in TMEM (tcgen05.st)
 //   O += P V      tcgen05.mma with A = P from TMEM, B = V from shared memory (MN-major)
 // Roles: warps 0-3 softmax + epilogue, warp 4 TMA producer, warp 5 MMA issuer / TMEM owner.
-// The grid is persistent; two blocks share an SM (256 TMEM columns each), so one block's
-// softmax overlaps the other's MMAs.  A small plan kernel turns the ragged layout into a
+// K and V tiles are double-buffered in shared memory and S in TMEM, so the next S = Q K^T is
+// issued while the softmax of the current tile runs.  The grid is persistent; two blocks
+// share an SM (256 TMEM columns each).  A small plan kernel turns the ragged layout into a
 // tile list.  Every mbarrier wait is bounded: on expiry the block records a timeout in the
 // workspace status word, unwinds, frees its TMEM and exits.
 #include "common.cuh"
@@ -21,11 +23,12 @@ namespace sp {
 using namespace ptx;
 
 constexpr int kBM = 128;              // query rows per tile
-constexpr int kBN = 128;              // keys per tile
+constexpr int kBN = 64;               // keys per tile
 constexpr int kHD = 128;              // head_dim
 constexpr int kTcThreads = 192;
-constexpr int kTileBytes = kBM * kHD * 2;
-constexpr int kTmemCols = 256;        // S/P: [0,128)  O: [128,256)
+constexpr int kQBytes = kBM * kHD * 2;     // 32 KB
+constexpr int kKVBytes = kBN * kHD * 2;    // 16 KB per stage
+constexpr int kTmemCols = 256;        // S/P double buffer: [0,64) [64,128)   O: [128,256)
 constexpr float kLog2eT = 1.4426950408889634f;
 constexpr float kLn2T = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.f;   // log2 units: rescale O only when the max grows by > 2^8
@@ -128,7 +131,7 @@ __global__ void __launch_bounds__(1024) prefill_plan_kernel(const PlanArgs a)
 // tile's last valid query row.
 struct KvTile {
     int row0;        // packed row of the first key
-    int n_valid;     // keys that exist (1..128)
+    int n_valid;     // keys that exist (1..kBN)
     int k_off;       // own-segment offset of the first key; -1 for preamble tiles (no causal limit)
 };
 __device__ __forceinline__ int n_kv_tiles(const TcTile &t)
@@ -148,20 +151,51 @@ __device__ __forceinline__ KvTile kv_tile(const TcTile &t, int j)
     return k;
 }
 
-enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_K_EMPTY, BAR_V_FULL, BAR_V_EMPTY, BAR_S_FULL, BAR_P_FULL,
-       BAR_O_DONE, BAR_COUNT };
+// Walks the block's work: items (query tile, head) in a grid-stride order, and inside an
+// item its key tiles.  g counts key tiles since the block started: it selects the ring
+// stage (g & 1) and the barrier parity ((g >> 1) & 1) of every double-buffered resource.
+struct Cursor {
+    const TcTile *tiles;
+    uint32_t it, n_items, stride, g, item_no;
+    int n_heads, h, j, n_kv;
+    TcTile t;
+    bool valid;
+    __device__ __forceinline__ void load()
+    {
+        valid = it < n_items;
+        if (valid) { t = tiles[it / n_heads]; h = it % n_heads; n_kv = n_kv_tiles(t); j = 0; }
+    }
+    __device__ __forceinline__ void init(const TcTile *tl, uint32_t n, int heads)
+    {
+        tiles = tl; n_items = n; n_heads = heads; it = blockIdx.x; stride = gridDim.x; g = 0; item_no = 0;
+        load();
+    }
+    __device__ __forceinline__ void next()
+    {
+        ++g;
+        if (++j == n_kv) { it += stride; ++item_no; load(); }
+    }
+    __device__ __forceinline__ bool last_of_item() const { return j == n_kv - 1; }
+};
+
+enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_K_EMPTY = BAR_K_FULL + 2, BAR_V_FULL = BAR_K_EMPTY + 2,
+       BAR_V_EMPTY = BAR_V_FULL + 2, BAR_S_FULL = BAR_V_EMPTY + 2, BAR_P_FULL = BAR_S_FULL + 2,
+       BAR_O_DONE = BAR_P_FULL + 2, BAR_COUNT };
 
 __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_constant__ TcParams p)
 {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    unsigned char *sQ = smem, *sK = smem + kTileBytes, *sV = smem + 2 * kTileBytes;
+    unsigned char *sQ = smem;                                   // 128 rows x 128 cols, two 64-col halves
+    unsigned char *sK = smem + kQBytes;                         // [2 stages] 64 keys x 128 cols
+    unsigned char *sV = sK + 2 * kKVBytes;                      // [2 stages]
+    unsigned char *sO = sV + 2 * kKVBytes;                      // [4 warps] 32 rows x 64 bytes, output staging
     __shared__ uint64_t bars[BAR_COUNT];
     __shared__ uint32_t tmem_base_s;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int i = 0; i < BAR_COUNT; ++i) mbar_init(&bars[i], i == BAR_P_FULL ? 128 : 1);
+        for (int i = 0; i < BAR_COUNT; ++i) mbar_init(&bars[i], (i == BAR_P_FULL || i == BAR_P_FULL + 1) ? 128 : 1);
         fence_mbar_init();
         prefetch_tmap(&p.mq); prefetch_tmap(&p.mk); prefetch_tmap(&p.mv);
     }
@@ -169,120 +203,141 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tb = tmem_base_s;
+    const uint32_t tb = tmem_base_s;                            // S0 [0,64) S1 [64,128) O [128,256)
     const uint32_t n_items = p.hdr->n_tiles * (uint32_t)p.n_heads;
     bool ok = true;
 
     if (warp == 4) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t qe = 0, ke = 0, ve = 0;
-            uint32_t nq = 0, nk = 0, nv = 0;          // loads issued per "full" barrier
-            for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
-                const TcTile t = p.tiles[it / p.n_heads];
-                const int h = it % p.n_heads, hk = h / p.kv_group;
-                if (!(ok = mbar_wait(&bars[BAR_Q_EMPTY], qe ^ 1))) break;
-                qe ^= 1;
-                mbar_expect_tx(&bars[BAR_Q_FULL], kTileBytes);
-                tma_load_2d(sQ, &p.mq, h * kHD, t.q_row, &bars[BAR_Q_FULL]);
-                tma_load_2d(sQ + kTileBytes / 2, &p.mq, h * kHD + 64, t.q_row, &bars[BAR_Q_FULL]);
-                ++nq;
-                const int n_kv = n_kv_tiles(t);
-                for (int j = 0; j < n_kv; ++j) {
-                    const KvTile kt = kv_tile(t, j);
-                    if (!(ok = mbar_wait(&bars[BAR_K_EMPTY], ke ^ 1))) break;
-                    ke ^= 1;
-                    mbar_expect_tx(&bars[BAR_K_FULL], kTileBytes);
-                    tma_load_2d(sK, &p.mk, hk * kHD, kt.row0, &bars[BAR_K_FULL]);
-                    tma_load_2d(sK + kTileBytes / 2, &p.mk, hk * kHD + 64, kt.row0, &bars[BAR_K_FULL]);
-                    ++nk;
-                    if (!(ok = mbar_wait(&bars[BAR_V_EMPTY], ve ^ 1))) break;
-                    ve ^= 1;
-                    mbar_expect_tx(&bars[BAR_V_FULL], kTileBytes);
-                    tma_load_2d(sV, &p.mv, hk * kHD, kt.row0, &bars[BAR_V_FULL]);
-                    tma_load_2d(sV + kTileBytes / 2, &p.mv, hk * kHD + 64, kt.row0, &bars[BAR_V_FULL]);
-                    ++nv;
+            uint32_t nq = 0, nk[2] = {0, 0}, nv[2] = {0, 0};     // loads issued per "full" barrier
+            Cursor c;
+            for (c.init(p.tiles, n_items, p.n_heads); c.valid && ok; c.next()) {
+                const int hk = c.h / p.kv_group;
+                if (c.j == 0) {
+                    if (!(ok = mbar_wait(&bars[BAR_Q_EMPTY], (c.item_no & 1) ^ 1))) break;
+                    mbar_expect_tx(&bars[BAR_Q_FULL], kQBytes);
+                    tma_load_2d(sQ, &p.mq, c.h * kHD, c.t.q_row, &bars[BAR_Q_FULL]);
+                    tma_load_2d(sQ + kQBytes / 2, &p.mq, c.h * kHD + 64, c.t.q_row, &bars[BAR_Q_FULL]);
+                    ++nq;
                 }
+                const KvTile kt = kv_tile(c.t, c.j);
+                const int st = c.g & 1;
+                const uint32_t ph = (c.g >> 1) & 1;
+                if (!(ok = mbar_wait(&bars[BAR_K_EMPTY + st], ph ^ 1))) break;
+                mbar_expect_tx(&bars[BAR_K_FULL + st], kKVBytes);
+                tma_load_2d(sK + st * kKVBytes, &p.mk, hk * kHD, kt.row0, &bars[BAR_K_FULL + st]);
+                tma_load_2d(sK + st * kKVBytes + kKVBytes / 2, &p.mk, hk * kHD + 64, kt.row0, &bars[BAR_K_FULL + st]);
+                ++nk[st];
+                if (!(ok = mbar_wait(&bars[BAR_V_EMPTY + st], ph ^ 1))) break;
+                mbar_expect_tx(&bars[BAR_V_FULL + st], kKVBytes);
+                tma_load_2d(sV + st * kKVBytes, &p.mv, hk * kHD, kt.row0, &bars[BAR_V_FULL + st]);
+                tma_load_2d(sV + st * kKVBytes + kKVBytes / 2, &p.mv, hk * kHD + 64, kt.row0, &bars[BAR_V_FULL + st]);
+                ++nv[st];
             }
             if (!ok) {
                 // a wait ran out: before the block may exit, its own copies in flight must
                 // have landed (bounded waits on the phase of the last load of each buffer)
                 if (nq) mbar_wait(&bars[BAR_Q_FULL], (nq - 1) & 1);
-                if (nk) mbar_wait(&bars[BAR_K_FULL], (nk - 1) & 1);
-                if (nv) mbar_wait(&bars[BAR_V_FULL], (nv - 1) & 1);
+                for (int st = 0; st < 2; ++st) {
+                    if (nk[st]) mbar_wait(&bars[BAR_K_FULL + st], (nk[st] - 1) & 1);
+                    if (nv[st]) mbar_wait(&bars[BAR_V_FULL + st], (nv[st] - 1) & 1);
+                }
             }
         }
         __syncwarp();
     } else if (warp == 5) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            uint32_t qf = 0, kf = 0, vf = 0, pf = 0;
             const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
-            for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
-                const TcTile t = p.tiles[it / p.n_heads];
-                if (!(ok = mbar_wait(&bars[BAR_Q_FULL], qf))) break;
-                qf ^= 1;
-                const int n_kv = n_kv_tiles(t);
-                for (int j = 0; j < n_kv; ++j) {
-                    const KvTile kt = kv_tile(t, j);
-                    const int n_mma = (kt.n_valid + 15) & ~15;
-                    if (!(ok = mbar_wait(&bars[BAR_K_FULL], kf))) break;
-                    kf ^= 1;
-                    tc_fence_after();
-                    const uint32_t id_s = idesc_bf16(kBM, n_mma, 0, 0);
+            const uint32_t id_o = idesc_bf16(kBM, kHD, 0, 1);
+            Cursor cs, cp;                      // cs: next S = Q K^T to issue; cp: next O += P V to issue
+            cs.init(p.tiles, n_items, p.n_heads);
+            cp.init(p.tiles, n_items, p.n_heads);
+
+            auto issue_s = [&](Cursor &c) -> bool {
+                const int st = c.g & 1;
+                if (c.j == 0 && !mbar_wait(&bars[BAR_Q_FULL], c.item_no & 1)) return false;
+                if (!mbar_wait(&bars[BAR_K_FULL + st], (c.g >> 1) & 1)) return false;
+                tc_fence_after();
+                const KvTile kt = kv_tile(c.t, c.j);
+                const int n_mma = (kt.n_valid + 15) & ~15;
+                const uint32_t id_s = idesc_bf16(kBM, n_mma, 0, 0);
 #pragma unroll
-                    for (int kk = 0; kk < kHD / 16; ++kk) {          // contraction over head_dim
-                        const uint32_t off = (kk >> 2) * (kTileBytes / 2) + (kk & 3) * 32;
-                        umma_ss(tb, smem_desc_sw128(aQ + off, 16, 1024), smem_desc_sw128(aK + off, 16, 1024), id_s, kk > 0);
-                    }
-                    umma_commit(&bars[BAR_S_FULL]);
-                    umma_commit(&bars[BAR_K_EMPTY]);
-                    if (j == n_kv - 1) umma_commit(&bars[BAR_Q_EMPTY]);
-                    if (!(ok = mbar_wait(&bars[BAR_P_FULL], pf))) break;
-                    pf ^= 1;
-                    if (!(ok = mbar_wait(&bars[BAR_V_FULL], vf))) break;
-                    vf ^= 1;
-                    tc_fence_after();
-                    const uint32_t id_o = idesc_bf16(kBM, kHD, 0, 1);
-                    for (int kk = 0; kk < n_mma / 16; ++kk)          // contraction over keys
-                        umma_ts(tb + 128, tb + kk * 8, smem_desc_sw128(aV + kk * 2048, kTileBytes / 2, 1024), id_o,
-                                (j > 0 || kk > 0) ? 1u : 0u);
-                    umma_commit(&bars[BAR_V_EMPTY]);
-                    if (j == n_kv - 1) umma_commit(&bars[BAR_O_DONE]);
+                for (int kk = 0; kk < kHD / 16; ++kk) {            // contraction over head_dim
+                    const uint32_t qo = (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32;
+                    const uint32_t ko = st * kKVBytes + (kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32;
+                    umma_ss(tb + st * kBN, smem_desc_sw128(aQ + qo, 16, 1024), smem_desc_sw128(aK + ko, 16, 1024), id_s, kk > 0);
                 }
+                umma_commit(&bars[BAR_S_FULL + st]);
+                umma_commit(&bars[BAR_K_EMPTY + st]);
+                if (c.last_of_item()) umma_commit(&bars[BAR_Q_EMPTY]);
+                c.next();
+                return true;
+            };
+
+            while (cp.valid && ok) {
+                if (cs.g == cp.g && !(ok = issue_s(cs))) break;       // S of the current tile
+                // S of the next tile, one ahead of the softmax, if its operands have landed
+                if (cs.valid && cs.g == cp.g + 1 &&
+                    (cs.j != 0 || mbar_test(&bars[BAR_Q_FULL], cs.item_no & 1)) &&
+                    mbar_test(&bars[BAR_K_FULL + (cs.g & 1)], (cs.g >> 1) & 1)) {
+                    if (!(ok = issue_s(cs))) break;
+                }
+                const int st = cp.g & 1;
+                const uint32_t ph = (cp.g >> 1) & 1;
+                const KvTile kt = kv_tile(cp.t, cp.j);
+                const int n_mma = (kt.n_valid + 15) & ~15;
+                if (!(ok = mbar_wait(&bars[BAR_P_FULL + st], ph))) break;
+                if (!(ok = mbar_wait(&bars[BAR_V_FULL + st], ph))) break;
+                tc_fence_after();
+                for (int kk = 0; kk < n_mma / 16; ++kk)               // contraction over keys
+                    umma_ts(tb + 128, tb + st * kBN + kk * 8,
+                            smem_desc_sw128(aV + st * kKVBytes + kk * 2048, kKVBytes / 2, 1024), id_o,
+                            (cp.j > 0 || kk > 0) ? 1u : 0u);
+                umma_commit(&bars[BAR_V_EMPTY + st]);
+                umma_commit(&bars[BAR_O_DONE]);
+                cp.next();
             }
         }
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ softmax + epilogue
-        uint32_t sf = 0, od = 0;
         const int row = warp * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
         const float sc = p.scale_log2e;
-        for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
-            const TcTile t = p.tiles[it / p.n_heads];
-            const int h = it % p.n_heads;
-            const int n_kv = n_kv_tiles(t);
+        unsigned char *stage = sO + warp * 2048;
+        Cursor c;
+        c.init(p.tiles, n_items, p.n_heads);
+        while (c.valid && ok) {
+            const TcTile t = c.t;
+            const int h = c.h, n_kv = c.n_kv;
             float m_ref = -INFINITY, l = 0.f;
-            for (int j = 0; j < n_kv; ++j) {
+            for (int j = 0; j < n_kv; ++j, c.next()) {
                 const KvTile kt = kv_tile(t, j);
+                const int st = c.g & 1;
+                const uint32_t s_addr = tb + lane_addr + st * kBN;
                 const int n_mma = (kt.n_valid + 15) & ~15;
-                const int n_chunks = (n_mma + 31) >> 5;
                 // visible keys of this row / of the warp's last row in this tile
                 const int lim = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + row - kt.k_off + 1);
                 const int wlim = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + warp * 32 + 31 - kt.k_off + 1);
-                if (!(ok = mbar_wait(&bars[BAR_S_FULL], sf))) break;
-                sf ^= 1;
+                if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
                 tc_fence_after();
 
+                uint32_t r0[32], r1[32];
+                const bool use0 = wlim > 0, use1 = wlim > 32;
+                if (use0) tmem_ld32(s_addr, r0);
+                if (use1) tmem_ld32(s_addr + 32, r1);
+                tmem_ld_wait();
+
                 float tmax = -INFINITY;
-                for (int c = 0; c < n_chunks && c * 32 < wlim; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(tb + lane_addr + c * 32, r);
-                    tmem_ld_wait();
+                if (use0) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        tmax = fmaxf(tmax, (c * 32 + i < lim) ? __uint_as_float(r[i]) : -INFINITY);
+                    for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, (i < lim) ? __uint_as_float(r0[i]) : -INFINITY);
+                }
+                if (use1) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, (32 + i < lim) ? __uint_as_float(r1[i]) : -INFINITY);
                 }
                 const float m_tile = tmax * sc;
                 float alpha = 1.f;
@@ -294,68 +349,95 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     m_ref = m_tile;
                     grow = true;
                 }
+                bool pv_seen = (j == 0);            // O += P V of the previous tile known complete?
                 if (__any_sync(0xffffffffu, grow)) {     // rare: bring O and l to the new reference
+                    if (!(ok = mbar_wait(&bars[BAR_O_DONE], (c.g - 1) & 1))) break;
+                    pv_seen = true;
+                    tc_fence_after();
                     l *= alpha;
-                    for (int c = 0; c < kHD / 32; ++c) {
+                    for (int cc = 0; cc < kHD / 32; ++cc) {
                         uint32_t r[32];
-                        tmem_ld32(tb + lane_addr + 128 + c * 32, r);
+                        tmem_ld32(tb + lane_addr + 128 + cc * 32, r);
                         tmem_ld_wait();
 #pragma unroll
                         for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                        tmem_st32(tb + lane_addr + 128 + c * 32, r);
+                        tmem_st32(tb + lane_addr + 128 + cc * 32, r);
                     }
                 }
-                for (int c = 0; c < n_chunks; ++c) {
+                {
                     uint32_t pk[16];
-                    if (c * 32 < wlim) {
-                        uint32_t r[32];
-                        tmem_ld32(tb + lane_addr + c * 32, r);
-                        tmem_ld_wait();
-                        float rs = 0.f;
+                    float rs = 0.f;
+                    if (use0) {
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
-                            const float x0 = fmaf(__uint_as_float(r[i]), sc, -m_ref);
-                            const float x1 = fmaf(__uint_as_float(r[i + 1]), sc, -m_ref);
-                            const float p0 = (c * 32 + i < lim) ? ex2(x0) : 0.f;
-                            const float p1 = (c * 32 + i + 1 < lim) ? ex2(x1) : 0.f;
+                            const float p0 = (i < lim) ? ex2(fmaf(__uint_as_float(r0[i]), sc, -m_ref)) : 0.f;
+                            const float p1 = (i + 1 < lim) ? ex2(fmaf(__uint_as_float(r0[i + 1]), sc, -m_ref)) : 0.f;
                             rs += p0 + p1;
                             pk[i >> 1] = pack_bf16x2(p0, p1);
                         }
-                        l += rs;
                     } else {
 #pragma unroll
                         for (int i = 0; i < 16; ++i) pk[i] = 0u;
                     }
-                    tmem_st16(tb + lane_addr + c * 16, pk);
+                    tmem_st16(s_addr, pk);
+                    if (n_mma > 32) {
+                        if (use1) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 2) {
+                                const float p0 = (32 + i < lim) ? ex2(fmaf(__uint_as_float(r1[i]), sc, -m_ref)) : 0.f;
+                                const float p1 = (33 + i < lim) ? ex2(fmaf(__uint_as_float(r1[i + 1]), sc, -m_ref)) : 0.f;
+                                rs += p0 + p1;
+                                pk[i >> 1] = pack_bf16x2(p0, p1);
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+                        }
+                        tmem_st16(s_addr + 16, pk);
+                    }
+                    l += rs;
                 }
+                // every completion of O += P V is observed exactly once, in order, so the
+                // barrier's parity stays unambiguous
+                if (!pv_seen && !(ok = mbar_wait(&bars[BAR_O_DONE], (c.g - 1) & 1))) break;
                 tmem_st_wait();
                 tc_fence_before();
-                mbar_arrive(&bars[BAR_P_FULL]);
+                mbar_arrive(&bars[BAR_P_FULL + st]);
             }
             if (!ok) break;
-            if (!(ok = mbar_wait(&bars[BAR_O_DONE], od))) break;
-            od ^= 1;
+            if (!(ok = mbar_wait(&bars[BAR_O_DONE], (c.g - 1) & 1))) break;     // last O += P V of the item
             tc_fence_after();
             const float inv = 1.f / l;
-            const bool live = row < t.n_rows;
-            __nv_bfloat16 *dst = p.out + ((int64_t)(t.q_row + row) * p.n_heads + h) * kHD;
-            for (int c = 0; c < kHD / 32; ++c) {
+            unsigned char *dst = reinterpret_cast<unsigned char *>(p.out) +
+                                 ((int64_t)t.q_row * p.n_heads + h) * (kHD * 2);
+            const int64_t row_pitch = (int64_t)p.n_heads * kHD * 2;
+            for (int cc = 0; cc < kHD / 32; ++cc) {
                 uint32_t r[32];
-                tmem_ld32(tb + lane_addr + 128 + c * 32, r);
+                tmem_ld32(tb + lane_addr + 128 + cc * 32, r);
                 tmem_ld_wait();
-                if (live) {
+                // thread = row -> shared staging (xor-swizzled 16-byte pieces) -> 8 rows x 64 contiguous
+                // bytes per store instruction
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
-                        w.y = pack_bf16x2(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-                        w.z = pack_bf16x2(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
-                        w.w = pack_bf16x2(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(dst + c * 32 + i) = w;
-                    }
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    uint4 w;
+                    w.x = pack_bf16x2(__uint_as_float(r[q4 * 8 + 0]) * inv, __uint_as_float(r[q4 * 8 + 1]) * inv);
+                    w.y = pack_bf16x2(__uint_as_float(r[q4 * 8 + 2]) * inv, __uint_as_float(r[q4 * 8 + 3]) * inv);
+                    w.z = pack_bf16x2(__uint_as_float(r[q4 * 8 + 4]) * inv, __uint_as_float(r[q4 * 8 + 5]) * inv);
+                    w.w = pack_bf16x2(__uint_as_float(r[q4 * 8 + 6]) * inv, __uint_as_float(r[q4 * 8 + 7]) * inv);
+                    *reinterpret_cast<uint4 *>(stage + lane * 64 + ((q4 ^ ((lane >> 1) & 3)) << 4)) = w;
                 }
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int rr = (lane >> 2) + 8 * i, piece = lane & 3;
+                    const uint4 w = *reinterpret_cast<const uint4 *>(stage + rr * 64 + ((piece ^ ((rr >> 1) & 3)) << 4));
+                    if (warp * 32 + rr < t.n_rows)
+                        *reinterpret_cast<uint4 *>(dst + (int64_t)(warp * 32 + rr) * row_pitch + cc * 64 + piece * 16) = w;
+                }
+                __syncwarp();
             }
-            if (live && p.lse) p.lse[(int64_t)h * p.total_tokens + t.q_row + row] = (m_ref + log2f(l)) * kLn2T;
+            if (row < t.n_rows && p.lse)
+                p.lse[(int64_t)h * p.total_tokens + t.q_row + row] = (m_ref + log2f(l)) * kLn2T;
             tc_fence_before();
         }
     }
@@ -371,12 +453,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-static int encode_rows_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int64_t rows, int64_t cols)
+static int encode_rows_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int64_t rows, int64_t cols, int box_rows)
 {
-    // [rows, cols] bf16 row-major; box = 128 rows x 64 columns (128 bytes), 128-byte swizzle
+    // [rows, cols] bf16 row-major; box = box_rows x 64 columns (128 bytes), 128-byte swizzle
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)kBM};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -412,9 +494,9 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
     SP_REQUIRE(((int64_t)n_heads * kHD * 2) % 16 == 0, SP_ERR_INVALID_ARG, "row stride must be a multiple of 16 bytes");
 
     TcParams p;
-    if (int rc = encode_rows_map(enc, &p.mq, q, lay->total_tokens, (int64_t)n_heads * kHD)) return rc;
-    if (int rc = encode_rows_map(enc, &p.mk, k, lay->total_tokens, (int64_t)n_kv_heads * kHD)) return rc;
-    if (int rc = encode_rows_map(enc, &p.mv, v, lay->total_tokens, (int64_t)n_kv_heads * kHD)) return rc;
+    if (int rc = encode_rows_map(enc, &p.mq, q, lay->total_tokens, (int64_t)n_heads * kHD, kBM)) return rc;
+    if (int rc = encode_rows_map(enc, &p.mk, k, lay->total_tokens, (int64_t)n_kv_heads * kHD, kBN)) return rc;
+    if (int rc = encode_rows_map(enc, &p.mv, v, lay->total_tokens, (int64_t)n_kv_heads * kHD, kBN)) return rc;
 
     TcHeader *hdr = static_cast<TcHeader *>(ws);
     TcTile *tiles = reinterpret_cast<TcTile *>(static_cast<char *>(ws) + 256);
@@ -436,7 +518,7 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
     const int64_t items = max_tiles(lay->n_prompts, lay->n_paths, lay->max_pre_len, lay->max_path_len) * n_heads;
     if (items == 0) return SP_OK;
     const int grid = (int)std::min<int64_t>(items, 2 * kNumSMs);
-    const int smem = 3 * kTileBytes + 1024;
+    const int smem = kQBytes + 4 * kKVBytes + 4 * 2048 + 1024;
     SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     prefill_tc_kernel<<<grid, kTcThreads, smem, st>>>(p);
     SP_CUDA(cudaGetLastError());

@@ -38,6 +38,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(kTryWaitHintNs) : "memory");
     return ok != 0;
 }
+// Non-blocking probe (no suspension).
+__device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait: false when the limit ran out (the caller records a timeout and unwinds).
 constexpr uint32_t kWaitLimit = 1u << 21;   // about two seconds at the hint above
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
