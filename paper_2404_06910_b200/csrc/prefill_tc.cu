@@ -157,13 +157,31 @@ __device__ __forceinline__ KvTile kv_tile(const TcTile &t, int j)
 struct Cursor {
     const TcTile *tiles;
     uint32_t it, n_items, stride, g, item_no;
-    int n_heads, h, j, n_kv;
+    int n_heads, h, j, n_kv, n_pre;
     TcTile t;
     bool valid;
     __device__ __forceinline__ void load()
     {
         valid = it < n_items;
-        if (valid) { t = tiles[it / n_heads]; h = it % n_heads; n_kv = n_kv_tiles(t); j = 0; }
+        if (valid) {
+            const uint32_t ti = it / (uint32_t)n_heads;
+            t = tiles[ti];
+            h = (int)(it - ti * (uint32_t)n_heads);
+            n_pre = (t.pre_len + kBN - 1) / kBN;
+            n_kv = n_pre + (t.q_off + t.n_rows + kBN - 1) / kBN;
+            j = 0;
+        }
+    }
+    __device__ __forceinline__ KvTile kv() const
+    {
+        KvTile k;
+        if (j < n_pre) {
+            k.row0 = t.pre_row + j * kBN; k.n_valid = min(kBN, t.pre_len - j * kBN); k.k_off = -1;
+        } else {
+            const int o = (j - n_pre) * kBN;
+            k.row0 = t.own_row + o; k.n_valid = min(kBN, t.q_off + t.n_rows - o); k.k_off = o;
+        }
+        return k;
     }
     __device__ __forceinline__ void init(const TcTile *tl, uint32_t n, int heads)
     {
@@ -221,7 +239,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     tma_load_2d(sQ + kQBytes / 2, &p.mq, c.h * kHD + 64, c.t.q_row, &bars[BAR_Q_FULL]);
                     ++nq;
                 }
-                const KvTile kt = kv_tile(c.t, c.j);
+                const KvTile kt = c.kv();
                 const int st = c.g & 1;
                 const uint32_t ph = (c.g >> 1) & 1;
                 if (!(ok = mbar_wait(&bars[BAR_K_EMPTY + st], ph ^ 1))) break;
@@ -249,26 +267,30 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
     } else if (warp == 5) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
+            // Descriptor words are loop-invariant up to a small address offset: build them once.
+            // High word: stride-dimension offset 1024 B (8-row groups), descriptor version 1, 128B swizzle.
+            const uint32_t d_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+            const uint32_t q_lo = ((smem_u32(sQ) & 0x3ffffu) >> 4) | (1u << 16);
+            const uint32_t k_lo = ((smem_u32(sK) & 0x3ffffu) >> 4) | (1u << 16);
+            const uint32_t v_lo = ((smem_u32(sV) & 0x3ffffu) >> 4) | ((uint32_t)((kKVBytes / 2) >> 4) << 16);
             const uint32_t id_o = idesc_bf16(kBM, kHD, 0, 1);
             Cursor cs, cp;                      // cs: next S = Q K^T to issue; cp: next O += P V to issue
             cs.init(p.tiles, n_items, p.n_heads);
             cp.init(p.tiles, n_items, p.n_heads);
 
             auto issue_s = [&](Cursor &c) -> bool {
-                const int st = c.g & 1;
+                const uint32_t st = c.g & 1;
                 if (c.j == 0 && !mbar_wait(&bars[BAR_Q_FULL], c.item_no & 1)) return false;
                 if (!mbar_wait(&bars[BAR_K_FULL + st], (c.g >> 1) & 1)) return false;
                 tc_fence_after();
-                const KvTile kt = kv_tile(c.t, c.j);
-                const int n_mma = (kt.n_valid + 15) & ~15;
-                const uint32_t id_s = idesc_bf16(kBM, n_mma, 0, 0);
+                const int n_mma = (c.kv().n_valid + 15) & ~15;
+                const uint32_t id_s = idesc_bf16(kBM, 0, 0, 0) | ((uint32_t)(n_mma >> 3) << 17);
+                const uint32_t kb = k_lo + st * (kKVBytes >> 4);
+                const uint32_t d = tb + st * kBN;
 #pragma unroll
-                for (int kk = 0; kk < kHD / 16; ++kk) {            // contraction over head_dim
-                    const uint32_t qo = (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32;
-                    const uint32_t ko = st * kKVBytes + (kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32;
-                    umma_ss(tb + st * kBN, smem_desc_sw128(aQ + qo, 16, 1024), smem_desc_sw128(aK + ko, 16, 1024), id_s, kk > 0);
-                }
+                for (int kk = 0; kk < kHD / 16; ++kk)              // contraction over head_dim
+                    umma_ss_lh(d, q_lo + (kk >> 2) * (kQBytes >> 5) + (kk & 3) * 2,
+                               kb + (kk >> 2) * (kKVBytes >> 5) + (kk & 3) * 2, d_hi, id_s, kk > 0 ? 1u : 0u);
                 umma_commit(&bars[BAR_S_FULL + st]);
                 umma_commit(&bars[BAR_K_EMPTY + st]);
                 if (c.last_of_item()) umma_commit(&bars[BAR_Q_EMPTY]);
@@ -284,17 +306,18 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     mbar_test(&bars[BAR_K_FULL + (cs.g & 1)], (cs.g >> 1) & 1)) {
                     if (!(ok = issue_s(cs))) break;
                 }
-                const int st = cp.g & 1;
+                const uint32_t st = cp.g & 1;
                 const uint32_t ph = (cp.g >> 1) & 1;
-                const KvTile kt = kv_tile(cp.t, cp.j);
-                const int n_mma = (kt.n_valid + 15) & ~15;
+                const int n_k = (cp.kv().n_valid + 15) >> 4;          // 16-key steps
                 if (!(ok = mbar_wait(&bars[BAR_P_FULL + st], ph))) break;
                 if (!(ok = mbar_wait(&bars[BAR_V_FULL + st], ph))) break;
                 tc_fence_after();
-                for (int kk = 0; kk < n_mma / 16; ++kk)               // contraction over keys
-                    umma_ts(tb + 128, tb + st * kBN + kk * 8,
-                            smem_desc_sw128(aV + st * kKVBytes + kk * 2048, kKVBytes / 2, 1024), id_o,
-                            (cp.j > 0 || kk > 0) ? 1u : 0u);
+                const uint32_t vb = v_lo + st * (kKVBytes >> 4);
+                const uint32_t pa = tb + st * kBN;
+#pragma unroll
+                for (int kk = 0; kk < kBN / 16; ++kk)                 // contraction over keys
+                    if (kk < n_k)
+                        umma_ts_lh(tb + 128, pa + kk * 8, vb + kk * (2048 >> 4), d_hi, id_o, (cp.j > 0 || kk > 0) ? 1u : 0u);
                 umma_commit(&bars[BAR_V_EMPTY + st]);
                 umma_commit(&bars[BAR_O_DONE]);
                 cp.next();
@@ -314,32 +337,40 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             const int h = c.h, n_kv = c.n_kv;
             float m_ref = -INFINITY, l = 0.f;
             for (int j = 0; j < n_kv; ++j, c.next()) {
-                const KvTile kt = kv_tile(t, j);
+                const KvTile kt = c.kv();
                 const int st = c.g & 1;
                 const uint32_t s_addr = tb + lane_addr + st * kBN;
                 const int n_mma = (kt.n_valid + 15) & ~15;
                 // visible keys of this row / of the warp's last row in this tile
                 const int lim = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + row - kt.k_off + 1);
-                const int wlim = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + warp * 32 + 31 - kt.k_off + 1);
                 if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
                 tc_fence_after();
 
+                // The row's scores stay in registers: one TMEM read per tile.
                 uint32_t r0[32], r1[32];
-                const bool use0 = wlim > 0, use1 = wlim > 32;
-                if (use0) tmem_ld32(s_addr, r0);
-                if (use1) tmem_ld32(s_addr + 32, r1);
+                const bool two = n_mma > 32;                     // uniform: second half of the tile in use
+                tmem_ld32(s_addr, r0);
+                if (two) tmem_ld32(s_addr + 32, r1);
                 tmem_ld_wait();
-
-                float tmax = -INFINITY;
-                if (use0) {
+                // keys past this row's limit (causal diagonal, ragged tail) -> -inf; skipped when
+                // the whole warp sees the whole tile
+                const int lim0 = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + warp * 32 - kt.k_off + 1);
+                if (lim0 < (two ? 64 : 32)) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, (i < lim) ? __uint_as_float(r0[i]) : -INFINITY);
-                }
-                if (use1) {
+                    for (int i = 0; i < 32; ++i) r0[i] = (i < lim) ? r0[i] : 0xff800000u;
+                    if (two) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, (32 + i < lim) ? __uint_as_float(r1[i]) : -INFINITY);
+                        for (int i = 0; i < 32; ++i) r1[i] = (32 + i < lim) ? r1[i] : 0xff800000u;
+                    }
                 }
-                const float m_tile = tmax * sc;
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(r0[i]));
+                if (two) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(r1[i]));
+                }
+                const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;
                 float alpha = 1.f;
                 bool grow = false;
                 if (j == 0) {
@@ -355,6 +386,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     pv_seen = true;
                     tc_fence_after();
                     l *= alpha;
+#pragma unroll 1
                     for (int cc = 0; cc < kHD / 32; ++cc) {
                         uint32_t r[32];
                         tmem_ld32(tb + lane_addr + 128 + cc * 32, r);
@@ -365,37 +397,29 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     }
                 }
                 {
+                    // masked scores are -inf, so exp2 gives exactly 0 for them
+                    const float nm = -m_ref;
+                    float rs[4] = {0.f, 0.f, 0.f, 0.f};
                     uint32_t pk[16];
-                    float rs = 0.f;
-                    if (use0) {
 #pragma unroll
-                        for (int i = 0; i < 32; i += 2) {
-                            const float p0 = (i < lim) ? ex2(fmaf(__uint_as_float(r0[i]), sc, -m_ref)) : 0.f;
-                            const float p1 = (i + 1 < lim) ? ex2(fmaf(__uint_as_float(r0[i + 1]), sc, -m_ref)) : 0.f;
-                            rs += p0 + p1;
-                            pk[i >> 1] = pack_bf16x2(p0, p1);
-                        }
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) pk[i] = 0u;
+                    for (int i = 0; i < 32; i += 2) {
+                        const float p0 = ex2(fmaf(__uint_as_float(r0[i]), sc, nm));
+                        const float p1 = ex2(fmaf(__uint_as_float(r0[i + 1]), sc, nm));
+                        rs[(i >> 1) & 3] += p0 + p1;
+                        pk[i >> 1] = pack_bf16x2(p0, p1);
                     }
                     tmem_st16(s_addr, pk);
-                    if (n_mma > 32) {
-                        if (use1) {
+                    if (two) {
 #pragma unroll
-                            for (int i = 0; i < 32; i += 2) {
-                                const float p0 = (32 + i < lim) ? ex2(fmaf(__uint_as_float(r1[i]), sc, -m_ref)) : 0.f;
-                                const float p1 = (33 + i < lim) ? ex2(fmaf(__uint_as_float(r1[i + 1]), sc, -m_ref)) : 0.f;
-                                rs += p0 + p1;
-                                pk[i >> 1] = pack_bf16x2(p0, p1);
-                            }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+                        for (int i = 0; i < 32; i += 2) {
+                            const float p0 = ex2(fmaf(__uint_as_float(r1[i]), sc, nm));
+                            const float p1 = ex2(fmaf(__uint_as_float(r1[i + 1]), sc, nm));
+                            rs[(i >> 1) & 3] += p0 + p1;
+                            pk[i >> 1] = pack_bf16x2(p0, p1);
                         }
                         tmem_st16(s_addr + 16, pk);
                     }
-                    l += rs;
+                    l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
                 }
                 // every completion of O += P V is observed exactly once, in order, so the
                 // barrier's parity stays unambiguous
@@ -411,30 +435,36 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             unsigned char *dst = reinterpret_cast<unsigned char *>(p.out) +
                                  ((int64_t)t.q_row * p.n_heads + h) * (kHD * 2);
             const int64_t row_pitch = (int64_t)p.n_heads * kHD * 2;
-            for (int cc = 0; cc < kHD / 32; ++cc) {
-                uint32_t r[32];
-                tmem_ld32(tb + lane_addr + 128 + cc * 32, r);
+#pragma unroll 1
+            for (int half = 0; half < 2; ++half) {
+                uint32_t ra[32], rb[32];
+                tmem_ld32(tb + lane_addr + 128 + half * 64, ra);
+                tmem_ld32(tb + lane_addr + 128 + half * 64 + 32, rb);
                 tmem_ld_wait();
-                // thread = row -> shared staging (xor-swizzled 16-byte pieces) -> 8 rows x 64 contiguous
-                // bytes per store instruction
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    uint4 w;
-                    w.x = pack_bf16x2(__uint_as_float(r[q4 * 8 + 0]) * inv, __uint_as_float(r[q4 * 8 + 1]) * inv);
-                    w.y = pack_bf16x2(__uint_as_float(r[q4 * 8 + 2]) * inv, __uint_as_float(r[q4 * 8 + 3]) * inv);
-                    w.z = pack_bf16x2(__uint_as_float(r[q4 * 8 + 4]) * inv, __uint_as_float(r[q4 * 8 + 5]) * inv);
-                    w.w = pack_bf16x2(__uint_as_float(r[q4 * 8 + 6]) * inv, __uint_as_float(r[q4 * 8 + 7]) * inv);
-                    *reinterpret_cast<uint4 *>(stage + lane * 64 + ((q4 ^ ((lane >> 1) & 3)) << 4)) = w;
-                }
-                __syncwarp();
+                for (int sub = 0; sub < 2; ++sub) {
+                    const uint32_t(&r)[32] = sub ? rb : ra;
+                    // thread = row -> shared staging (xor-swizzled 16-byte pieces) -> each store
+                    // instruction writes 8 rows x 64 contiguous bytes
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int rr = (lane >> 2) + 8 * i, piece = lane & 3;
-                    const uint4 w = *reinterpret_cast<const uint4 *>(stage + rr * 64 + ((piece ^ ((rr >> 1) & 3)) << 4));
-                    if (warp * 32 + rr < t.n_rows)
-                        *reinterpret_cast<uint4 *>(dst + (int64_t)(warp * 32 + rr) * row_pitch + cc * 64 + piece * 16) = w;
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(r[q4 * 8 + 0]) * inv, __uint_as_float(r[q4 * 8 + 1]) * inv);
+                        w.y = pack_bf16x2(__uint_as_float(r[q4 * 8 + 2]) * inv, __uint_as_float(r[q4 * 8 + 3]) * inv);
+                        w.z = pack_bf16x2(__uint_as_float(r[q4 * 8 + 4]) * inv, __uint_as_float(r[q4 * 8 + 5]) * inv);
+                        w.w = pack_bf16x2(__uint_as_float(r[q4 * 8 + 6]) * inv, __uint_as_float(r[q4 * 8 + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(stage + lane * 64 + ((q4 ^ ((lane >> 1) & 3)) << 4)) = w;
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int rr = (lane >> 2) + 8 * i, piece = lane & 3;
+                        const uint4 w = *reinterpret_cast<const uint4 *>(stage + rr * 64 + ((piece ^ ((rr >> 1) & 3)) << 4));
+                        if (warp * 32 + rr < t.n_rows)
+                            *reinterpret_cast<uint4 *>(dst + (int64_t)(warp * 32 + rr) * row_pitch + (half * 2 + sub) * 64 + piece * 16) = w;
+                    }
+                    __syncwarp();
                 }
-                __syncwarp();
             }
             if (row < t.n_rows && p.lse)
                 p.lse[(int64_t)h * p.total_tokens + t.q_row + row] = (m_ref + log2f(l)) * kLn2T;
