@@ -196,9 +196,10 @@ struct Cursor {
     __device__ __forceinline__ bool last_of_item() const { return j == n_kv - 1; }
 };
 
-enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_K_EMPTY = BAR_K_FULL + 2, BAR_V_FULL = BAR_K_EMPTY + 2,
-       BAR_V_EMPTY = BAR_V_FULL + 2, BAR_S_FULL = BAR_V_EMPTY + 2, BAR_P_FULL = BAR_S_FULL + 2,
-       BAR_O_DONE = BAR_P_FULL + 2, BAR_COUNT };
+// S_FULL[st] (S = Q K^T of a tile complete) also tells the producer that K stage st is free;
+// O_DONE[st] (O += P V complete) also frees V stage st: one tcgen05.commit serves both waiters.
+enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_V_FULL = BAR_K_FULL + 2, BAR_S_FULL = BAR_V_FULL + 2,
+       BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2, BAR_COUNT = BAR_O_DONE + 2 };
 
 __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_constant__ TcParams p)
 {
@@ -242,12 +243,12 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 const KvTile kt = c.kv();
                 const int st = c.g & 1;
                 const uint32_t ph = (c.g >> 1) & 1;
-                if (!(ok = mbar_wait(&bars[BAR_K_EMPTY + st], ph ^ 1))) break;
+                if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], ph ^ 1))) break;       // K stage free
                 mbar_expect_tx(&bars[BAR_K_FULL + st], kKVBytes);
                 tma_load_2d(sK + st * kKVBytes, &p.mk, hk * kHD, kt.row0, &bars[BAR_K_FULL + st]);
                 tma_load_2d(sK + st * kKVBytes + kKVBytes / 2, &p.mk, hk * kHD + 64, kt.row0, &bars[BAR_K_FULL + st]);
                 ++nk[st];
-                if (!(ok = mbar_wait(&bars[BAR_V_EMPTY + st], ph ^ 1))) break;
+                if (!(ok = mbar_wait(&bars[BAR_O_DONE + st], ph ^ 1))) break;       // V stage free
                 mbar_expect_tx(&bars[BAR_V_FULL + st], kKVBytes);
                 tma_load_2d(sV + st * kKVBytes, &p.mv, hk * kHD, kt.row0, &bars[BAR_V_FULL + st]);
                 tma_load_2d(sV + st * kKVBytes + kKVBytes / 2, &p.mv, hk * kHD + 64, kt.row0, &bars[BAR_V_FULL + st]);
@@ -278,34 +279,29 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             cs.init(p.tiles, n_items, p.n_heads);
             cp.init(p.tiles, n_items, p.n_heads);
 
-            auto issue_s = [&](Cursor &c) -> bool {
-                const uint32_t st = c.g & 1;
-                if (c.j == 0 && !mbar_wait(&bars[BAR_Q_FULL], c.item_no & 1)) return false;
-                if (!mbar_wait(&bars[BAR_K_FULL + st], (c.g >> 1) & 1)) return false;
-                tc_fence_after();
-                const int n_mma = (c.kv().n_valid + 15) & ~15;
-                const uint32_t id_s = idesc_bf16(kBM, 0, 0, 0) | ((uint32_t)(n_mma >> 3) << 17);
-                const uint32_t kb = k_lo + st * (kKVBytes >> 4);
-                const uint32_t d = tb + st * kBN;
-#pragma unroll
-                for (int kk = 0; kk < kHD / 16; ++kk)              // contraction over head_dim
-                    umma_ss_lh(d, q_lo + (kk >> 2) * (kQBytes >> 5) + (kk & 3) * 2,
-                               kb + (kk >> 2) * (kKVBytes >> 5) + (kk & 3) * 2, d_hi, id_s, kk > 0 ? 1u : 0u);
-                umma_commit(&bars[BAR_S_FULL + st]);
-                umma_commit(&bars[BAR_K_EMPTY + st]);
-                if (c.last_of_item()) umma_commit(&bars[BAR_Q_EMPTY]);
-                c.next();
-                return true;
-            };
-
             while (cp.valid && ok) {
-                if (cs.g == cp.g && !(ok = issue_s(cs))) break;       // S of the current tile
-                // S of the next tile, one ahead of the softmax, if its operands have landed
-                if (cs.valid && cs.g == cp.g + 1 &&
-                    (cs.j != 0 || mbar_test(&bars[BAR_Q_FULL], cs.item_no & 1)) &&
-                    mbar_test(&bars[BAR_K_FULL + (cs.g & 1)], (cs.g >> 1) & 1)) {
-                    if (!(ok = issue_s(cs))) break;
+                // S = Q K^T: the current tile's must be issued; the next tile's is issued one
+                // ahead of the softmax as soon as its operands have landed
+                while (cs.valid && (cs.g == cp.g ||
+                                    (cs.g == cp.g + 1 && (cs.j != 0 || mbar_test(&bars[BAR_Q_FULL], cs.item_no & 1)) &&
+                                     mbar_test(&bars[BAR_K_FULL + (cs.g & 1)], (cs.g >> 1) & 1)))) {
+                    const uint32_t st = cs.g & 1;
+                    if (cs.j == 0 && !(ok = mbar_wait(&bars[BAR_Q_FULL], cs.item_no & 1))) break;
+                    if (!(ok = mbar_wait(&bars[BAR_K_FULL + st], (cs.g >> 1) & 1))) break;
+                    tc_fence_after();
+                    const int n_mma = (cs.kv().n_valid + 15) & ~15;
+                    const uint32_t id_s = idesc_bf16(kBM, 0, 0, 0) | ((uint32_t)(n_mma >> 3) << 17);
+                    const uint32_t kb = k_lo + st * (kKVBytes >> 4);
+                    const uint32_t d = tb + st * kBN;
+#pragma unroll
+                    for (int kk = 0; kk < kHD / 16; ++kk)              // contraction over head_dim
+                        umma_ss_lh(d, q_lo + (kk >> 2) * (kQBytes >> 5) + (kk & 3) * 2,
+                                   kb + (kk >> 2) * (kKVBytes >> 5) + (kk & 3) * 2, d_hi, id_s, kk > 0 ? 1u : 0u);
+                    umma_commit(&bars[BAR_S_FULL + st]);
+                    if (cs.last_of_item()) umma_commit(&bars[BAR_Q_EMPTY]);
+                    cs.next();
                 }
+                if (!ok) break;
                 const uint32_t st = cp.g & 1;
                 const uint32_t ph = (cp.g >> 1) & 1;
                 const int n_k = (cp.kv().n_valid + 15) >> 4;          // 16-key steps
@@ -318,8 +314,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 for (int kk = 0; kk < kBN / 16; ++kk)                 // contraction over keys
                     if (kk < n_k)
                         umma_ts_lh(tb + 128, pa + kk * 8, vb + kk * (2048 >> 4), d_hi, id_o, (cp.j > 0 || kk > 0) ? 1u : 0u);
-                umma_commit(&bars[BAR_V_EMPTY + st]);
-                umma_commit(&bars[BAR_O_DONE]);
+                umma_commit(&bars[BAR_O_DONE + st]);
                 cp.next();
             }
         }
@@ -332,17 +327,26 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
         unsigned char *stage = sO + warp * 2048;
         Cursor c;
         c.init(p.tiles, n_items, p.n_heads);
-        while (c.valid && ok) {
-            const TcTile t = c.t;
-            const int h = c.h, n_kv = c.n_kv;
-            float m_ref = -INFINITY, l = 0.f;
-            for (int j = 0; j < n_kv; ++j, c.next()) {
+        float m_ref = -INFINITY, l = 0.f;          // running reference maximum (log2 units) and row sum
+        // A finished item whose output is still in TMEM: its epilogue runs after the softmax of
+        // the next item's first tile, so the wait for its last O += P V is hidden behind work.
+        bool have_prev = false;
+        TcTile prev_t = {};
+        int prev_h = 0;
+        float prev_m = 0.f, prev_l = 1.f;
+
+        while ((c.valid || have_prev) && ok) {
+            const int st = c.g & 1;
+            const bool first = c.valid && c.j == 0;
+            if (c.valid) {
+                const TcTile &t = c.t;
                 const KvTile kt = c.kv();
-                const int st = c.g & 1;
                 const uint32_t s_addr = tb + lane_addr + st * kBN;
                 const int n_mma = (kt.n_valid + 15) & ~15;
-                // visible keys of this row / of the warp's last row in this tile
+                // visible keys of this row / of the warp's first row in this tile
                 const int lim = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + row - kt.k_off + 1);
+                const int lim0 = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + warp * 32 - kt.k_off + 1);
+                if (first) { m_ref = -INFINITY; l = 0.f; }
                 if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
                 tc_fence_after();
 
@@ -354,7 +358,6 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 tmem_ld_wait();
                 // keys past this row's limit (causal diagonal, ragged tail) -> -inf; skipped when
                 // the whole warp sees the whole tile
-                const int lim0 = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + warp * 32 - kt.k_off + 1);
                 if (lim0 < (two ? 64 : 32)) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) r0[i] = (i < lim) ? r0[i] : 0xff800000u;
@@ -373,17 +376,17 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;
                 float alpha = 1.f;
                 bool grow = false;
-                if (j == 0) {
+                if (first) {
                     m_ref = m_tile;
                 } else if (m_tile > m_ref + kRescaleThreshold) {
                     alpha = ex2(m_ref - m_tile);
                     m_ref = m_tile;
                     grow = true;
                 }
-                bool pv_seen = (j == 0);            // O += P V of the previous tile known complete?
                 if (__any_sync(0xffffffffu, grow)) {     // rare: bring O and l to the new reference
-                    if (!(ok = mbar_wait(&bars[BAR_O_DONE], (c.g - 1) & 1))) break;
-                    pv_seen = true;
+                    // needs the previous tile's O += P V complete; it is observed again below,
+                    // which returns at once (same phase)
+                    if (!(ok = mbar_wait(&bars[BAR_O_DONE + ((c.g - 1) & 1)], ((c.g - 1) >> 1) & 1))) break;
                     tc_fence_after();
                     l *= alpha;
 #pragma unroll 1
@@ -421,54 +424,64 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     }
                     l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
                 }
-                // every completion of O += P V is observed exactly once, in order, so the
-                // barrier's parity stays unambiguous
-                if (!pv_seen && !(ok = mbar_wait(&bars[BAR_O_DONE], (c.g - 1) & 1))) break;
-                tmem_st_wait();
-                tc_fence_before();
-                mbar_arrive(&bars[BAR_P_FULL + st]);
             }
-            if (!ok) break;
-            if (!(ok = mbar_wait(&bars[BAR_O_DONE], (c.g - 1) & 1))) break;     // last O += P V of the item
-            tc_fence_after();
-            const float inv = 1.f / l;
-            unsigned char *dst = reinterpret_cast<unsigned char *>(p.out) +
-                                 ((int64_t)t.q_row * p.n_heads + h) * (kHD * 2);
-            const int64_t row_pitch = (int64_t)p.n_heads * kHD * 2;
+            // Every completion of O += P V is observed exactly once per stage, in order (tile
+            // g - 1 here), so the barrier parity stays unambiguous.
+            if (c.g > 0 && !(ok = mbar_wait(&bars[BAR_O_DONE + ((c.g - 1) & 1)], ((c.g - 1) >> 1) & 1))) break;
+
+            if (have_prev && (first || !c.valid)) {
+                // ---- epilogue of the previous item: O / l -> bf16 -> global
+                tc_fence_after();
+                const float inv = 1.f / prev_l;
+                unsigned char *dst = reinterpret_cast<unsigned char *>(p.out) +
+                                     ((int64_t)prev_t.q_row * p.n_heads + prev_h) * (kHD * 2);
+                const int64_t row_pitch = (int64_t)p.n_heads * kHD * 2;
 #pragma unroll 1
-            for (int half = 0; half < 2; ++half) {
-                uint32_t ra[32], rb[32];
-                tmem_ld32(tb + lane_addr + 128 + half * 64, ra);
-                tmem_ld32(tb + lane_addr + 128 + half * 64 + 32, rb);
-                tmem_ld_wait();
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t ra[32], rb[32];
+                    tmem_ld32(tb + lane_addr + 128 + half * 64, ra);
+                    tmem_ld32(tb + lane_addr + 128 + half * 64 + 32, rb);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int sub = 0; sub < 2; ++sub) {
-                    const uint32_t(&r)[32] = sub ? rb : ra;
-                    // thread = row -> shared staging (xor-swizzled 16-byte pieces) -> each store
-                    // instruction writes 8 rows x 64 contiguous bytes
+                    for (int sub = 0; sub < 2; ++sub) {
+                        // thread = row -> shared staging (xor-swizzled 16-byte pieces) -> each store
+                        // instruction writes 8 rows x 64 contiguous bytes
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(r[q4 * 8 + 0]) * inv, __uint_as_float(r[q4 * 8 + 1]) * inv);
-                        w.y = pack_bf16x2(__uint_as_float(r[q4 * 8 + 2]) * inv, __uint_as_float(r[q4 * 8 + 3]) * inv);
-                        w.z = pack_bf16x2(__uint_as_float(r[q4 * 8 + 4]) * inv, __uint_as_float(r[q4 * 8 + 5]) * inv);
-                        w.w = pack_bf16x2(__uint_as_float(r[q4 * 8 + 6]) * inv, __uint_as_float(r[q4 * 8 + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(stage + lane * 64 + ((q4 ^ ((lane >> 1) & 3)) << 4)) = w;
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            uint4 w;
+                            const uint32_t *r = sub ? rb : ra;
+                            w.x = pack_bf16x2(__uint_as_float(r[q4 * 8 + 0]) * inv, __uint_as_float(r[q4 * 8 + 1]) * inv);
+                            w.y = pack_bf16x2(__uint_as_float(r[q4 * 8 + 2]) * inv, __uint_as_float(r[q4 * 8 + 3]) * inv);
+                            w.z = pack_bf16x2(__uint_as_float(r[q4 * 8 + 4]) * inv, __uint_as_float(r[q4 * 8 + 5]) * inv);
+                            w.w = pack_bf16x2(__uint_as_float(r[q4 * 8 + 6]) * inv, __uint_as_float(r[q4 * 8 + 7]) * inv);
+                            *reinterpret_cast<uint4 *>(stage + lane * 64 + ((q4 ^ ((lane >> 1) & 3)) << 4)) = w;
+                        }
+                        __syncwarp();
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int rr = (lane >> 2) + 8 * i, piece = lane & 3;
+                            const uint4 w = *reinterpret_cast<const uint4 *>(stage + rr * 64 + ((piece ^ ((rr >> 1) & 3)) << 4));
+                            if (warp * 32 + rr < prev_t.n_rows)
+                                *reinterpret_cast<uint4 *>(dst + (int64_t)(warp * 32 + rr) * row_pitch + (half * 2 + sub) * 64 + piece * 16) = w;
+                        }
+                        __syncwarp();
                     }
-                    __syncwarp();
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int rr = (lane >> 2) + 8 * i, piece = lane & 3;
-                        const uint4 w = *reinterpret_cast<const uint4 *>(stage + rr * 64 + ((piece ^ ((rr >> 1) & 3)) << 4));
-                        if (warp * 32 + rr < t.n_rows)
-                            *reinterpret_cast<uint4 *>(dst + (int64_t)(warp * 32 + rr) * row_pitch + (half * 2 + sub) * 64 + piece * 16) = w;
-                    }
-                    __syncwarp();
                 }
+                if (row < prev_t.n_rows && p.lse)
+                    p.lse[(int64_t)prev_h * p.total_tokens + prev_t.q_row + row] = (prev_m + log2f(prev_l)) * kLn2T;
+                have_prev = false;
             }
-            if (row < t.n_rows && p.lse)
-                p.lse[(int64_t)h * p.total_tokens + t.q_row + row] = (m_ref + log2f(l)) * kLn2T;
+            if (!c.valid) break;
+
+            // P of this tile is in TMEM (and O of the previous item has been read out): release
+            // the tile to the MMA issuer
+            tmem_st_wait();
             tc_fence_before();
+            mbar_arrive(&bars[BAR_P_FULL + st]);
+            if (c.last_of_item()) {
+                have_prev = true; prev_t = c.t; prev_h = c.h; prev_m = m_ref; prev_l = l;
+            }
+            c.next();
         }
     }
 
