@@ -5,11 +5,12 @@
 // (all visible) followed by the segment's own rows up to the diagonal; key tiles that the
 // fork-join mask excludes are never loaded or multiplied.  Per key tile of up to 64 keys:
 //   S = Q K^T     tcgen05.mma, A and B from TMA-staged 128B-swizzled shared memory, fp32 in TMEM
-//   P = softmax   4 warps, one thread per query row (tcgen05.ld, the row stays in registers),
+//   P = softmax   8 warps, two threads per query row (tcgen05.ld, scores stay in registers),
 //                 online max / sum with lazy rescaling, P rounded to bf16 and written over S
 //                 in TMEM (tcgen05.st)
 //   O += P V      tcgen05.mma with A = P from TMEM, B = V from shared memory (MN-major)
-// Roles: warps 0-3 softmax + epilogue, warp 4 TMA producer, warp 5 MMA issuer / TMEM owner.
+// Roles: warps 0-7 softmax + epilogue (two threads per query row, 32 keys of a tile each),
+// warp 8 TMA producer, warp 9 MMA issuer / TMEM owner.
 // K and V tiles are double-buffered in shared memory and S in TMEM, so the next S = Q K^T is
 // issued while the softmax of the current tile runs.  The grid is persistent; two blocks
 // share an SM (256 TMEM columns each).  A small plan kernel turns the ragged layout into a
@@ -25,7 +26,8 @@ using namespace ptx;
 constexpr int kBM = 128;              // query rows per tile
 constexpr int kBN = 64;               // keys per tile
 constexpr int kHD = 128;              // head_dim
-constexpr int kTcThreads = 192;
+constexpr int kSoftmaxWarps = 8;      // two threads per query row: each owns 32 of a tile's 64 keys
+constexpr int kTcThreads = (kSoftmaxWarps + 2) * 32;
 constexpr int kQBytes = kBM * kHD * 2;     // 32 KB
 constexpr int kKVBytes = kBN * kHD * 2;    // 16 KB per stage
 constexpr int kTmemCols = 256;        // S/P double buffer: [0,64) [64,128)   O: [128,256)
@@ -134,23 +136,6 @@ struct KvTile {
     int n_valid;     // keys that exist (1..kBN)
     int k_off;       // own-segment offset of the first key; -1 for preamble tiles (no causal limit)
 };
-__device__ __forceinline__ int n_kv_tiles(const TcTile &t)
-{
-    return (t.pre_len + kBN - 1) / kBN + (t.q_off + t.n_rows + kBN - 1) / kBN;
-}
-__device__ __forceinline__ KvTile kv_tile(const TcTile &t, int j)
-{
-    const int n_pre = (t.pre_len + kBN - 1) / kBN;
-    KvTile k;
-    if (j < n_pre) {
-        k.row0 = t.pre_row + j * kBN; k.n_valid = min(kBN, t.pre_len - j * kBN); k.k_off = -1;
-    } else {
-        const int o = (j - n_pre) * kBN;
-        k.row0 = t.own_row + o; k.n_valid = min(kBN, t.q_off + t.n_rows - o); k.k_off = o;
-    }
-    return k;
-}
-
 // Walks the block's work: items (query tile, head) in a grid-stride order, and inside an
 // item its key tiles.  g counts key tiles since the block started: it selects the ring
 // stage (g & 1) and the barrier parity ((g >> 1) & 1) of every double-buffered resource.
@@ -198,8 +183,12 @@ struct Cursor {
 
 // S_FULL[st] (S = Q K^T of a tile complete) also tells the producer that K stage st is free;
 // O_DONE[st] (O += P V complete) also frees V stage st: one tcgen05.commit serves both waiters.
+// X_MAX[parity] / X_SUM: the two threads of a row exchange their half-row maximum (per
+// tile) and half-row sum (per item) through shared memory; mbarriers rather than bar.sync so
+// that these waits are bounded like all others.
 enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_V_FULL = BAR_K_FULL + 2, BAR_S_FULL = BAR_V_FULL + 2,
-       BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2, BAR_COUNT = BAR_O_DONE + 2 };
+       BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2, BAR_X_MAX = BAR_O_DONE + 2,
+       BAR_X_SUM = BAR_X_MAX + 2, BAR_COUNT };
 
 __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_constant__ TcParams p)
 {
@@ -208,17 +197,19 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
     unsigned char *sQ = smem;                                   // 128 rows x 128 cols, two 64-col halves
     unsigned char *sK = smem + kQBytes;                         // [2 stages] 64 keys x 128 cols
     unsigned char *sV = sK + 2 * kKVBytes;                      // [2 stages]
-    unsigned char *sO = sV + 2 * kKVBytes;                      // [4 warps] 32 rows x 64 bytes, output staging
+    unsigned char *sO = sV + 2 * kKVBytes;                      // [8 warps] 32 rows x 32 bytes, output staging
     __shared__ uint64_t bars[BAR_COUNT];
     __shared__ uint32_t tmem_base_s;
+    __shared__ float x_max[2][2][kBM];                          // [tile parity][half][row]
+    __shared__ float x_sum[2][2][kBM];                          // [item parity][half][row]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int i = 0; i < BAR_COUNT; ++i) mbar_init(&bars[i], (i == BAR_P_FULL || i == BAR_P_FULL + 1) ? 128 : 1);
+        for (int i = 0; i < BAR_COUNT; ++i) mbar_init(&bars[i], (i >= BAR_P_FULL && i < BAR_P_FULL + 2) || i >= BAR_X_MAX ? kSoftmaxWarps * 32 : 1);
         fence_mbar_init();
         prefetch_tmap(&p.mq); prefetch_tmap(&p.mk); prefetch_tmap(&p.mv);
     }
-    if (warp == 5) { tmem_alloc(&tmem_base_s, kTmemCols); tmem_relinquish(); }
+    if (warp == kSoftmaxWarps + 1) { tmem_alloc(&tmem_base_s, kTmemCols); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -226,7 +217,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
     const uint32_t n_items = p.hdr->n_tiles * (uint32_t)p.n_heads;
     bool ok = true;
 
-    if (warp == 4) {
+    if (warp == kSoftmaxWarps) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t nq = 0, nk[2] = {0, 0}, nv[2] = {0, 0};     // loads issued per "full" barrier
@@ -265,7 +256,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             }
         }
         __syncwarp();
-    } else if (warp == 5) {
+    } else if (warp == kSoftmaxWarps + 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             // Descriptor words are loop-invariant up to a small address offset: build them once.
@@ -321,18 +312,23 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ softmax + epilogue
-        const int row = warp * 32 + lane;
-        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        // Thread (row, hf): TMEM lanes are reachable by warp % 4, so warps w and w + 4 share the
+        // same 32 rows; hf = warp / 4 picks keys [32 hf, 32 hf + 32) of every 64-key tile and
+        // output columns [64 hf, 64 hf + 64).
+        const int quad = warp & 3, hf = warp >> 2;
+        const int row = quad * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         const float sc = p.scale_log2e;
-        unsigned char *stage = sO + warp * 2048;
+        unsigned char *stage = sO + warp * 1024;
         Cursor c;
         c.init(p.tiles, n_items, p.n_heads);
-        float m_ref = -INFINITY, l = 0.f;          // running reference maximum (log2 units) and row sum
+        float m_ref = -INFINITY, l = 0.f;          // reference maximum (log2 units), this thread's half of the row sum
         // A finished item whose output is still in TMEM: its epilogue runs after the softmax of
         // the next item's first tile, so the wait for its last O += P V is hidden behind work.
         bool have_prev = false;
         TcTile prev_t = {};
         int prev_h = 0;
+        uint32_t prev_no = 0;
         float prev_m = 0.f, prev_l = 1.f;
 
         while ((c.valid || have_prev) && ok) {
@@ -341,39 +337,41 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             if (c.valid) {
                 const TcTile &t = c.t;
                 const KvTile kt = c.kv();
-                const uint32_t s_addr = tb + lane_addr + st * kBN;
+                const uint32_t s_addr = tb + lane_addr + st * kBN + hf * 32;
                 const int n_mma = (kt.n_valid + 15) & ~15;
-                // visible keys of this row / of the warp's first row in this tile
-                const int lim = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + row - kt.k_off + 1);
-                const int lim0 = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + warp * 32 - kt.k_off + 1);
+                // keys of my 32 that this row / the warp's first and last rows may see
+                const int vis = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + row - kt.k_off + 1);
+                const int vis0 = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + quad * 32 - kt.k_off + 1);
+                const int vis31 = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + quad * 32 + 31 - kt.k_off + 1);
+                const int lim = vis - hf * 32;
+                const bool in_use = hf * 32 < n_mma;             // uniform: my columns are read by O += P V
+                const bool any_vis = vis31 - hf * 32 > 0;         // uniform: some row of the warp sees some key of mine
                 if (first) { m_ref = -INFINITY; l = 0.f; }
                 if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
                 tc_fence_after();
 
-                // The row's scores stay in registers: one TMEM read per tile.
-                uint32_t r0[32], r1[32];
-                const bool two = n_mma > 32;                     // uniform: second half of the tile in use
-                tmem_ld32(s_addr, r0);
-                if (two) tmem_ld32(s_addr + 32, r1);
-                tmem_ld_wait();
-                // keys past this row's limit (causal diagonal, ragged tail) -> -inf; skipped when
-                // the whole warp sees the whole tile
-                if (lim0 < (two ? 64 : 32)) {
+                // My half of the row's scores stays in registers: one TMEM read per tile.
+                uint32_t r[32];
+                float hmax = -INFINITY;
+                if (any_vis) {
+                    tmem_ld32(s_addr, r);
+                    tmem_ld_wait();
+                    // keys past the row's limit (causal diagonal, ragged tail) -> -inf; skipped
+                    // when the whole warp sees all 32
+                    if (vis0 - hf * 32 < 32) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) r0[i] = (i < lim) ? r0[i] : 0xff800000u;
-                    if (two) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) r1[i] = (32 + i < lim) ? r1[i] : 0xff800000u;
+                        for (int i = 0; i < 32; ++i) r[i] = (i < lim) ? r[i] : 0xff800000u;
                     }
-                }
-                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(r0[i]));
-                if (two) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(r1[i]));
+                    for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(r[i]));
+                    hmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
                 }
-                const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;
+                // exchange the half-row maxima
+                x_max[st][hf][row] = hmax;
+                mbar_arrive(&bars[BAR_X_MAX + st]);
+                if (!(ok = mbar_wait(&bars[BAR_X_MAX + st], (c.g >> 1) & 1))) break;
+                const float m_tile = fmaxf(hmax, x_max[st][hf ^ 1][row]) * sc;
                 float alpha = 1.f;
                 bool grow = false;
                 if (first) {
@@ -390,39 +388,34 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     tc_fence_after();
                     l *= alpha;
 #pragma unroll 1
-                    for (int cc = 0; cc < kHD / 32; ++cc) {
-                        uint32_t r[32];
-                        tmem_ld32(tb + lane_addr + 128 + cc * 32, r);
+                    for (int cc = 0; cc < 2; ++cc) {
+                        uint32_t o[32];
+                        tmem_ld32(tb + lane_addr + 128 + hf * 64 + cc * 32, o);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                        tmem_st32(tb + lane_addr + 128 + cc * 32, r);
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(tb + lane_addr + 128 + hf * 64 + cc * 32, o);
                     }
                 }
-                {
-                    // masked scores are -inf, so exp2 gives exactly 0 for them
-                    const float nm = -m_ref;
-                    float rs[4] = {0.f, 0.f, 0.f, 0.f};
+                if (in_use) {
                     uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        const float p0 = ex2(fmaf(__uint_as_float(r0[i]), sc, nm));
-                        const float p1 = ex2(fmaf(__uint_as_float(r0[i + 1]), sc, nm));
-                        rs[(i >> 1) & 3] += p0 + p1;
-                        pk[i >> 1] = pack_bf16x2(p0, p1);
-                    }
-                    tmem_st16(s_addr, pk);
-                    if (two) {
+                    if (any_vis) {
+                        // masked scores are -inf, so exp2 gives exactly 0 for them
+                        const float nm = -m_ref;
+                        float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
-                            const float p0 = ex2(fmaf(__uint_as_float(r1[i]), sc, nm));
-                            const float p1 = ex2(fmaf(__uint_as_float(r1[i + 1]), sc, nm));
+                            const float p0 = ex2(fmaf(__uint_as_float(r[i]), sc, nm));
+                            const float p1 = ex2(fmaf(__uint_as_float(r[i + 1]), sc, nm));
                             rs[(i >> 1) & 3] += p0 + p1;
                             pk[i >> 1] = pack_bf16x2(p0, p1);
                         }
-                        tmem_st16(s_addr + 16, pk);
+                        l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) pk[i] = 0u;
                     }
-                    l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
+                    tmem_st16(tb + lane_addr + st * kBN + hf * 16, pk);
                 }
             }
             // Every completion of O += P V is observed exactly once per stage, in order (tile
@@ -430,45 +423,49 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             if (c.g > 0 && !(ok = mbar_wait(&bars[BAR_O_DONE + ((c.g - 1) & 1)], ((c.g - 1) >> 1) & 1))) break;
 
             if (have_prev && (first || !c.valid)) {
-                // ---- epilogue of the previous item: O / l -> bf16 -> global
+                // ---- epilogue of the previous item: O / l -> bf16 -> global (my 64 columns)
                 tc_fence_after();
-                const float inv = 1.f / prev_l;
+                const int xp = prev_no & 1;
+                x_sum[xp][hf][row] = prev_l;
+                mbar_arrive(&bars[BAR_X_SUM]);
+                if (!(ok = mbar_wait(&bars[BAR_X_SUM], xp))) break;
+                const float l_row = prev_l + x_sum[xp][hf ^ 1][row];
+                const float inv = 1.f / l_row;
                 unsigned char *dst = reinterpret_cast<unsigned char *>(p.out) +
-                                     ((int64_t)prev_t.q_row * p.n_heads + prev_h) * (kHD * 2);
+                                     ((int64_t)prev_t.q_row * p.n_heads + prev_h) * (kHD * 2) + hf * 128;
                 const int64_t row_pitch = (int64_t)p.n_heads * kHD * 2;
 #pragma unroll 1
-                for (int half = 0; half < 2; ++half) {
-                    uint32_t ra[32], rb[32];
-                    tmem_ld32(tb + lane_addr + 128 + half * 64, ra);
-                    tmem_ld32(tb + lane_addr + 128 + half * 64 + 32, rb);
+                for (int cc = 0; cc < 2; ++cc) {
+                    uint32_t ro[32];
+                    tmem_ld32(tb + lane_addr + 128 + hf * 64 + cc * 32, ro);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int sub = 0; sub < 2; ++sub) {
+                    for (int sub = 0; sub < 2; ++sub) {      // 16 output columns (32 bytes per row) per round
                         // thread = row -> shared staging (xor-swizzled 16-byte pieces) -> each store
-                        // instruction writes 8 rows x 64 contiguous bytes
+                        // instruction writes 16 rows x 32 contiguous bytes
 #pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4) {
+                        for (int q2 = 0; q2 < 2; ++q2) {
+                            const int e = sub * 16 + q2 * 8;
                             uint4 w;
-                            const uint32_t *r = sub ? rb : ra;
-                            w.x = pack_bf16x2(__uint_as_float(r[q4 * 8 + 0]) * inv, __uint_as_float(r[q4 * 8 + 1]) * inv);
-                            w.y = pack_bf16x2(__uint_as_float(r[q4 * 8 + 2]) * inv, __uint_as_float(r[q4 * 8 + 3]) * inv);
-                            w.z = pack_bf16x2(__uint_as_float(r[q4 * 8 + 4]) * inv, __uint_as_float(r[q4 * 8 + 5]) * inv);
-                            w.w = pack_bf16x2(__uint_as_float(r[q4 * 8 + 6]) * inv, __uint_as_float(r[q4 * 8 + 7]) * inv);
-                            *reinterpret_cast<uint4 *>(stage + lane * 64 + ((q4 ^ ((lane >> 1) & 3)) << 4)) = w;
+                            w.x = pack_bf16x2(__uint_as_float(ro[e + 0]) * inv, __uint_as_float(ro[e + 1]) * inv);
+                            w.y = pack_bf16x2(__uint_as_float(ro[e + 2]) * inv, __uint_as_float(ro[e + 3]) * inv);
+                            w.z = pack_bf16x2(__uint_as_float(ro[e + 4]) * inv, __uint_as_float(ro[e + 5]) * inv);
+                            w.w = pack_bf16x2(__uint_as_float(ro[e + 6]) * inv, __uint_as_float(ro[e + 7]) * inv);
+                            *reinterpret_cast<uint4 *>(stage + lane * 32 + ((q2 ^ ((lane >> 2) & 1)) << 4)) = w;
                         }
                         __syncwarp();
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int rr = (lane >> 2) + 8 * i, piece = lane & 3;
-                            const uint4 w = *reinterpret_cast<const uint4 *>(stage + rr * 64 + ((piece ^ ((rr >> 1) & 3)) << 4));
-                            if (warp * 32 + rr < prev_t.n_rows)
-                                *reinterpret_cast<uint4 *>(dst + (int64_t)(warp * 32 + rr) * row_pitch + (half * 2 + sub) * 64 + piece * 16) = w;
+                        for (int i = 0; i < 2; ++i) {
+                            const int rr = (lane >> 1) + 16 * i, piece = lane & 1;
+                            const uint4 w = *reinterpret_cast<const uint4 *>(stage + rr * 32 + ((piece ^ ((rr >> 2) & 1)) << 4));
+                            if (quad * 32 + rr < prev_t.n_rows)
+                                *reinterpret_cast<uint4 *>(dst + (int64_t)(quad * 32 + rr) * row_pitch + (cc * 2 + sub) * 32 + piece * 16) = w;
                         }
                         __syncwarp();
                     }
                 }
-                if (row < prev_t.n_rows && p.lse)
-                    p.lse[(int64_t)prev_h * p.total_tokens + prev_t.q_row + row] = (prev_m + log2f(prev_l)) * kLn2T;
+                if (hf == 0 && row < prev_t.n_rows && p.lse)
+                    p.lse[(int64_t)prev_h * p.total_tokens + prev_t.q_row + row] = (prev_m + log2f(l_row)) * kLn2T;
                 have_prev = false;
             }
             if (!c.valid) break;
@@ -479,7 +476,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             tc_fence_before();
             mbar_arrive(&bars[BAR_P_FULL + st]);
             if (c.last_of_item()) {
-                have_prev = true; prev_t = c.t; prev_h = c.h; prev_m = m_ref; prev_l = l;
+                have_prev = true; prev_t = c.t; prev_h = c.h; prev_m = m_ref; prev_l = l; prev_no = c.item_no;
             }
             c.next();
         }
@@ -488,7 +485,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
     if (!ok && lane == 0) atomicExch(p.status, (uint32_t)STATUS_TIMEOUT);
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) tmem_dealloc(tb, kTmemCols);
+    if (warp == kSoftmaxWarps + 1) tmem_dealloc(tb, kTmemCols);
 }
 
 // ---- host side ---------------------------------------------------------------------------
@@ -561,7 +558,7 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
     const int64_t items = max_tiles(lay->n_prompts, lay->n_paths, lay->max_pre_len, lay->max_path_len) * n_heads;
     if (items == 0) return SP_OK;
     const int grid = (int)std::min<int64_t>(items, 2 * kNumSMs);
-    const int smem = kQBytes + 4 * kKVBytes + 4 * 2048 + 1024;
+    const int smem = kQBytes + 4 * kKVBytes + kSoftmaxWarps * 1024 + 1024;
     SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     prefill_tc_kernel<<<grid, kTcThreads, smem, st>>>(p);
     SP_CUDA(cudaGetLastError());
