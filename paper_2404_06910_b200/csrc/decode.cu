@@ -12,7 +12,7 @@
 namespace sp {
 
 constexpr int kDecThreads = 128;
-constexpr int kDecUnroll = 8;        // keys in flight per key group
+constexpr int kDecUnroll = 4;        // keys in flight per key group (kept small: occupancy hides latency better)
 constexpr int kDecMaxSplits = 64;
 constexpr float kLog2eD = 1.4426950408889634f;
 constexpr float kLn2D = 0.6931471805599453f;
@@ -70,7 +70,7 @@ template <> struct Raw16<float> {
 };
 
 template <typename T, int D>
-__global__ void __launch_bounds__(kDecThreads, 5)
+__global__ void __launch_bounds__(kDecThreads, 8)
 decode_kernel(const __grid_constant__ DecodeArgs a)
 {
     constexpr int N = Vec<T>::N;            // elements per 16-byte load
