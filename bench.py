@@ -36,9 +36,9 @@ from workloads import (draw_decode_inputs, draw_lengths, draw_logits, draw_prior
 METRIC = "superposition prefill useful TFLOP/s over the whole hot-path step"
 UNIT = "TFLOP/s"
 PREFILL_LAUNCHES = 2           # kernels sp_superpose_prefill launches per call (tile plan + attention)
-# dram__bytes_read.sum + dram__bytes_write.sum of one prefill launch, from the ncu capture
-# summarised under profiles/ (None until captured for the current kernel).
-NCU_PREFILL_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch, (kernel, workload) -> bytes, from
+# the ncu captures summarised under profiles/ (absent = not captured for the current kernel).
+NCU_TRAFFIC_BYTES = {}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -168,6 +168,7 @@ class HotPath:
         # per decode step rope x2 + decode
         self.launches = 2 + PREFILL_LAUNCHES + 2 + 1 + self.steps_dec * 3
         self.decode_graph = None
+        self.kv_sets = [(self.k, self.v)]
 
     def decode_bytes(self):
         kept = self.kept.cpu().numpy()
@@ -213,14 +214,26 @@ class HotPath:
             self.decode_loop()
         mark()
 
-    def decode_loop(self):
+    def make_kv_sets(self, l2_bytes):
+        """A decode step reads only the kept paths' KV (about 100 MB on the smaller workloads),
+        which would stay in the 126 MB L2 if every step re-read the same buffers.  A real
+        model has one cache per layer, so consecutive decode launches read different memory:
+        rotate over enough copies of the cache to exceed twice the L2."""
+        keys = self.lay.max_pre_len + self.cfg.top_k * float(np.mean(self.lay.doc_len + self.lay.qry_len))
+        per_step = max(1.0, self.B * keys * 2 * self.Hkv * self.D * self.cfg.elt_bytes)
+        n = int(min(8, max(1, math.ceil(2.0 * l2_bytes / per_step))))
+        self.kv_sets = [(self.k, self.v)] + [(self.k.clone(), self.v.clone()) for _ in range(n - 1)]
+
+    def decode_loop(self, with_rope=True):
         sp, cfg = self.sp, self.cfg
         H, Hkv, D, B = self.H, self.Hkv, self.D, self.B
         ld = self.steps_dec * Hkv * D
         for t in range(self.steps_dec):
-            sp.sp_rope_apply(self.dq[t], self.tpos[t], H, D, base=cfg.rope_base)
-            sp.sp_rope_apply(self.tk[:, t], self.tpos[t], Hkv, D, n_tokens=B, ld_token=ld, base=cfg.rope_base)
-            sp.sp_pruned_decode(self.dq[t], self.k, self.v, self.dl, self.kept, cfg.top_k, self.tk, self.tv,
+            if with_rope:
+                sp.sp_rope_apply(self.dq[t], self.tpos[t], H, D, base=cfg.rope_base)
+                sp.sp_rope_apply(self.tk[:, t], self.tpos[t], Hkv, D, n_tokens=B, ld_token=ld, base=cfg.rope_base)
+            kc, vc = self.kv_sets[t % len(self.kv_sets)]
+            sp.sp_pruned_decode(self.dq[t], kc, vc, self.dl, self.kept, cfg.top_k, self.tk, self.tv,
                                 self.tail_len[t], self.steps_dec, self.scale, self.dec_out[t], None, self.ws_dec)
 
     def capture_decode_graph(self):
@@ -258,10 +271,11 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=device)
     cfg = get_config(args.workload)
     hp = HotPath(cfg, cfg.seed + 1000 * rank, sp, device, args.prompts, args.decode_steps)
+    l2_bytes = torch.cuda.get_device_properties(device).L2_cache_size
+    hp.make_kv_sets(l2_bytes)
     if not args.no_graph:
         hp.capture_decode_graph()
     peaks = load_peaks()
-    l2_bytes = torch.cuda.get_device_properties(device).L2_cache_size
     flush = None
     if hp.bytes_prefill < 2 * l2_bytes:          # small workload: flush L2 between steps
         flush = torch.empty(2 * l2_bytes, dtype=torch.uint8, device=device)
@@ -291,6 +305,15 @@ def run_ours(args):
             flush.zero_()
     sync()
     clocks = sampler.stop() if rank == 0 else None
+
+    # decode kernel alone (no rope launches), eager, for the per-launch roofline of that kernel
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    hp.decode_loop(with_rope=False)
+    d0.record()
+    hp.decode_loop(with_rope=False)
+    d1.record()
+    sync()
+    decode_kernel_ms = d0.elapsed_time(d1) / hp.steps_dec
 
     stage_ms = np.zeros(len(STAGES))
     total_ms = 0.0
@@ -340,8 +363,25 @@ def run_ours(args):
             "topk": {"ms": ms["topk"]},
             "decode": {"ms": ms["decode"], "steps": hp.steps_dec, "gbs": gb(hp.bytes_decode, ms["decode"]),
                        "frac_hbm": gb(hp.bytes_decode, ms["decode"]) / peaks["hbm_gbs"],
+                       "kernel_only_ms_per_launch": decode_kernel_ms,
+                       "kernel_only_gbs": gb(hp.bytes_decode / hp.steps_dec, decode_kernel_ms),
+                       "kernel_only_frac_hbm": gb(hp.bytes_decode / hp.steps_dec, decode_kernel_ms) / peaks["hbm_gbs"],
+                       "kv_sets": len(hp.kv_sets),
                        "includes": "2 rope launches + 1 decode launch per token" + ("" if args.no_graph else ", replayed from a CUDA graph")},
         }
+        roof_prefill = {"kernel": "prefill_tc_kernel (sp_superpose_prefill)", "bound": "hbm", "achieved": pre_gbs,
+                        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": pre_gbs / peaks["hbm_gbs"],
+                        "traffic": NCU_TRAFFIC_BYTES.get(("prefill", cfg.name)), "peak_source": peaks["source"],
+                        "algorithmic_bytes": hp.bytes_prefill, "launch_ms": ms["prefill"], "useful_tflops": pre_tf,
+                        "frac_bf16_sustained": pre_tf / peaks["bf16_tflops_sustained"]}
+        dec_gbs = gb(hp.bytes_decode / hp.steps_dec, decode_kernel_ms)
+        roof_decode = {"kernel": "decode_kernel (sp_pruned_decode)", "bound": "hbm", "achieved": dec_gbs,
+                       "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"],
+                       "traffic": NCU_TRAFFIC_BYTES.get(("decode", cfg.name)), "peak_source": peaks["source"],
+                       "algorithmic_bytes": hp.bytes_decode / hp.steps_dec, "launch_ms": decode_kernel_ms,
+                       "launches_per_step": hp.steps_dec}
+        # the dominant kernel = the one with the largest total device time in a step
+        roofline = roof_decode if decode_kernel_ms * hp.steps_dec > ms["prefill"] else roof_prefill
         line = {
             "metric": METRIC, "value": world * tf(hp.flop_prefill, ms_per_step), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
@@ -349,14 +389,11 @@ def run_ours(args):
             "dtype": cfg.dtype, "data": "synthetic",
             "config": {"workload": cfg.name, "prompts_per_gpu": hp.B, "paths": hp.lay.n_paths,
                        "tokens": hp.lay.total_tokens, "heads": hp.H, "head_dim": hp.D, "vocab": cfg.vocab,
-                       "top_k": cfg.top_k, "decode_steps": hp.steps_dec, "allowed_pairs": hp.pairs,
+                       "top_k": cfg.top_k, "decode_steps": hp.steps_dec, "allowed_pairs": hp.pairs, "decode_kv_sets": len(hp.kv_sets),
                        "l2": "inputs larger than L2" if flush is None else "L2 flushed between steps",
                        "parallelism": f"dp{world} (independent prompts per GPU, no collective)"},
-            "roofline": {"kernel": "sp_superpose_prefill", "bound": "hbm", "achieved": pre_gbs,
-                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": pre_gbs / peaks["hbm_gbs"],
-                         "traffic": NCU_PREFILL_TRAFFIC_BYTES.get(cfg.name), "peak_source": peaks["source"],
-                         "algorithmic_bytes": hp.bytes_prefill, "useful_tflops": pre_tf,
-                         "frac_bf16_sustained": pre_tf / peaks["bf16_tflops_sustained"]},
+            "roofline": roofline,
+            "roofline_prefill": roof_prefill,
             "kernels": kernels,
             "e2e": None if not e2e_steps else {
                 "value": world * tf(hp.flop_prefill, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,

@@ -44,7 +44,7 @@ static size_t decode_counter_bytes(int n_prompts, int n_heads)
 static int decode_split_cap(int n_prompts, int n_heads)
 {
     const int64_t bh = std::max<int64_t>(1, (int64_t)n_prompts * n_heads);
-    const int64_t want = (8LL * kNumSMs + bh - 1) / bh;
+    const int64_t want = (8LL * kNumSMs) / bh;      // 8 blocks per SM: all blocks of a launch are resident at once
     return (int)std::min<int64_t>(kDecMaxSplits, std::max<int64_t>(1, want));
 }
 
