@@ -46,6 +46,24 @@ NCU_TRAFFIC_BYTES = {
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+def rank_seed(cfg, rank: int) -> int:
+    """Every rank draws its own prompts (data parallel over independent prompts)."""
+    return cfg.seed + 1000 * rank
+
+
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Per-rank timings -> the slowest rank's (the job's) timings, on every rank."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def aggregate_value(flop_per_rank: float, ms: float, world: int) -> float:
+    """Whole-job useful TFLOP/s: every rank does flop_per_rank in the (max-over-ranks) time."""
+    return world * flop_per_rank / (ms * 1e-3) / 1e12
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -274,7 +292,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
     cfg = get_config(args.workload)
-    hp = HotPath(cfg, cfg.seed + 1000 * rank, sp, device, args.prompts, args.decode_steps)
+    hp = HotPath(cfg, rank_seed(cfg, rank), sp, device, args.prompts, args.decode_steps)
     l2_bytes = torch.cuda.get_device_properties(device).L2_cache_size
     hp.make_kv_sets(l2_bytes)
     if not args.no_graph:
@@ -344,10 +362,7 @@ def run_ours(args):
         sync()
         e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
-    t = torch.tensor([ms_per_step, e2e_ms], dtype=torch.float64, device=device)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_per_step, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step, e2e_ms = max_over_ranks([ms_per_step, e2e_ms], dist, device)
 
     if rank == 0:
         tf = lambda flop, ms: flop / (ms * 1e-3) / 1e12
@@ -387,7 +402,7 @@ def run_ours(args):
         # the dominant kernel = the one with the largest total device time in a step
         roofline = roof_decode if decode_kernel_ms * hp.steps_dec > ms["prefill"] else roof_prefill
         line = {
-            "metric": METRIC, "value": world * tf(hp.flop_prefill, ms_per_step), "unit": UNIT,
+            "metric": METRIC, "value": aggregate_value(hp.flop_prefill, ms_per_step, world), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": cfg.dtype, "data": "synthetic",
@@ -400,7 +415,7 @@ def run_ours(args):
             "roofline_prefill": roof_prefill,
             "kernels": kernels,
             "e2e": None if not e2e_steps else {
-                "value": world * tf(hp.flop_prefill, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
+                "value": aggregate_value(hp.flop_prefill, e2e_ms, world), "unit": UNIT, "ms_per_step": e2e_ms,
                 "steps": e2e_steps, "h2d_bytes_per_step": bi, "d2h_bytes_per_step": bo},
             "gpu_launches": hp.launches * args.steps,
             "clocks": clocks,

@@ -16,6 +16,8 @@
 // share an SM (256 TMEM columns each).  A small plan kernel turns the ragged layout into a
 // tile list.  Every mbarrier wait is bounded: on expiry the block records a timeout in the
 // workspace status word, unwinds, frees its TMEM and exits.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "tc_ptx.cuh"
 
@@ -66,6 +68,7 @@ struct TcParams {
     int n_heads, kv_group;
     int64_t total_tokens;
     float scale_log2e;
+    int stall_producer;               // test hook: the producer issues no load, so every wait runs out
 };
 
 // ---- plan: ragged layout -> tile list ---------------------------------------------------
@@ -188,7 +191,7 @@ struct Cursor {
 // that these waits are bounded like all others.
 enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_V_FULL = BAR_K_FULL + 2, BAR_S_FULL = BAR_V_FULL + 2,
        BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2, BAR_X_MAX = BAR_O_DONE + 2,
-       BAR_X_SUM = BAR_X_MAX + 2, BAR_COUNT };
+       BAR_X_SUM = BAR_X_MAX + 2, BAR_DRAIN, BAR_COUNT };
 
 __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_constant__ TcParams p)
 {
@@ -205,7 +208,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int i = 0; i < BAR_COUNT; ++i) mbar_init(&bars[i], (i >= BAR_P_FULL && i < BAR_P_FULL + 2) || i >= BAR_X_MAX ? kSoftmaxWarps * 32 : 1);
+        for (int i = 0; i < BAR_COUNT; ++i) mbar_init(&bars[i], (i >= BAR_P_FULL && i < BAR_P_FULL + 2) || (i >= BAR_X_MAX && i <= BAR_X_SUM) ? kSoftmaxWarps * 32 : 1);
         fence_mbar_init();
         prefetch_tmap(&p.mq); prefetch_tmap(&p.mk); prefetch_tmap(&p.mv);
     }
@@ -222,7 +225,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
         if (lane == 0) {
             uint32_t nq = 0, nk[2] = {0, 0}, nv[2] = {0, 0};     // loads issued per "full" barrier
             Cursor c;
-            for (c.init(p.tiles, n_items, p.n_heads); c.valid && ok; c.next()) {
+            for (c.init(p.tiles, n_items, p.n_heads); c.valid && ok && !p.stall_producer; c.next()) {
                 const int hk = c.h / p.kv_group;
                 if (c.j == 0) {
                     if (!(ok = mbar_wait(&bars[BAR_Q_EMPTY], (c.item_no & 1) ^ 1))) break;
@@ -307,6 +310,12 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                         umma_ts_lh(tb + 128, pa + kk * 8, vb + kk * (2048 >> 4), d_hi, id_o, (cp.j > 0 || kk > 0) ? 1u : 0u);
                 umma_commit(&bars[BAR_O_DONE + st]);
                 cp.next();
+            }
+            if (!ok) {
+                // a wait ran out: let every MMA already issued finish (bounded) before the
+                // tensor memory they write is freed
+                umma_commit(&bars[BAR_DRAIN]);
+                mbar_wait(&bars[BAR_DRAIN], 0);
             }
         }
         __syncwarp();
@@ -554,6 +563,11 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
     p.out = static_cast<__nv_bfloat16 *>(out); p.lse = lse;
     p.n_heads = n_heads; p.kv_group = n_heads / n_kv_heads;
     p.total_tokens = lay->total_tokens; p.scale_log2e = scale * kLog2eT;
+    // Failure-detection test hook (host-injected, no GPU fault): with SP_TEST_STALL_PRODUCER=1 in
+    // the environment no tile is ever loaded, every bounded wait expires, the blocks unwind and
+    // the call reports SP_ERR_TIMEOUT through the workspace status word.
+    const char *stall = std::getenv("SP_TEST_STALL_PRODUCER");
+    p.stall_producer = (stall && stall[0] == '1') ? 1 : 0;
 
     const int64_t items = max_tiles(lay->n_prompts, lay->n_paths, lay->max_pre_len, lay->max_path_len) * n_heads;
     if (items == 0) return SP_OK;
