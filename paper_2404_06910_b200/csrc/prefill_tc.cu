@@ -353,8 +353,11 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 const int vis0 = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + quad * 32 - kt.k_off + 1);
                 const int vis31 = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + quad * 32 + 31 - kt.k_off + 1);
                 const int lim = vis - hf * 32;
-                const bool in_use = hf * 32 < n_mma;             // uniform: my columns are read by O += P V
-                const bool any_vis = vis31 - hf * 32 > 0;         // uniform: some row of the warp sees some key of mine
+                // A warp whose 32 rows lie past the tile's last valid row does no arithmetic at all:
+                // its rows of P and O are never stored (it still takes part in every barrier).
+                const bool live_w = quad * 32 < t.n_rows;
+                const bool in_use = live_w && hf * 32 < n_mma;   // uniform: my part of P is read by O += P V and matters
+                const bool any_vis = live_w && vis31 - hf * 32 > 0;   // uniform: some row of the warp sees some key of mine
                 if (first) { m_ref = -INFINITY; l = 0.f; }
                 if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
                 tc_fence_after();
@@ -440,6 +443,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 if (!(ok = mbar_wait(&bars[BAR_X_SUM], xp))) break;
                 const float l_row = prev_l + x_sum[xp][hf ^ 1][row];
                 const float inv = 1.f / l_row;
+                if (quad * 32 < prev_t.n_rows) {
                 unsigned char *dst = reinterpret_cast<unsigned char *>(p.out) +
                                      ((int64_t)prev_t.q_row * p.n_heads + prev_h) * (kHD * 2) + hf * 128;
                 const int64_t row_pitch = (int64_t)p.n_heads * kHD * 2;
@@ -475,6 +479,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 }
                 if (hf == 0 && row < prev_t.n_rows && p.lse)
                     p.lse[(int64_t)prev_h * p.total_tokens + prev_t.q_row + row] = (prev_m + log2f(l_row)) * kLn2T;
+                }
                 have_prev = false;
             }
             if (!c.valid) break;
