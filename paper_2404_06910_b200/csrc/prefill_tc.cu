@@ -410,24 +410,31 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     }
                 }
                 if (in_use) {
-                    uint32_t pk[16];
+                    const uint32_t p_addr = tb + lane_addr + st * kBN + hf * 16;
                     if (any_vis) {
                         // masked scores are -inf, so exp2 gives exactly 0 for them
                         const float nm = -m_ref;
                         float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                        for (int i = 0; i < 32; i += 2) {
-                            const float p0 = ex2(fmaf(__uint_as_float(r[i]), sc, nm));
-                            const float p1 = ex2(fmaf(__uint_as_float(r[i + 1]), sc, nm));
-                            rs[(i >> 1) & 3] += p0 + p1;
-                            pk[i >> 1] = pack_bf16x2(p0, p1);
+                        for (int q8 = 0; q8 < 2; ++q8) {          // 16 keys -> 8 packed pairs per store
+                            uint32_t pk[8];
+#pragma unroll
+                            for (int i = 0; i < 16; i += 2) {
+                                const float p0 = ex2(fmaf(__uint_as_float(r[q8 * 16 + i]), sc, nm));
+                                const float p1 = ex2(fmaf(__uint_as_float(r[q8 * 16 + i + 1]), sc, nm));
+                                rs[(i >> 1) & 3] += p0 + p1;
+                                pk[i >> 1] = pack_bf16x2(p0, p1);
+                            }
+                            tmem_st8(p_addr + q8 * 8, pk);
                         }
                         l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
                     } else {
+                        uint32_t z[8];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) pk[i] = 0u;
+                        for (int i = 0; i < 8; ++i) z[i] = 0u;
+                        tmem_st8(p_addr, z);
+                        tmem_st8(p_addr + 8, z);
                     }
-                    tmem_st16(tb + lane_addr + st * kBN + hf * 16, pk);
                 }
             }
             // Every completion of O += P V is observed exactly once per stage, in order (tile
