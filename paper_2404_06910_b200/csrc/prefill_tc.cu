@@ -5,12 +5,13 @@
 // (all visible) followed by the segment's own rows up to the diagonal; key tiles that the
 // fork-join mask excludes are never loaded or multiplied.  Per key tile of up to 64 keys:
 //   S = Q K^T     tcgen05.mma, A and B from TMA-staged 128B-swizzled shared memory, fp32 in TMEM
-//   P = softmax   8 warps, two threads per query row (tcgen05.ld, scores stay in registers),
-//                 online max / sum with lazy rescaling, P rounded to bf16 and written over S
-//                 in TMEM (tcgen05.st)
+//   P = softmax   4 warps, one thread per query row (tcgen05.ld, the tile's scores stay in
+//                 registers), online max / sum with lazy rescaling, P rounded to bf16 and written
+//                 over S in TMEM (tcgen05.st)
 //   O += P V      tcgen05.mma with A = P from TMEM, B = V from shared memory (MN-major)
-// Roles: warps 0-7 softmax + epilogue (two threads per query row, 32 keys of a tile each),
-// warp 8 TMA producer, warp 9 MMA issuer / TMEM owner.
+// Roles (warpgroups of 4 warps, registers rebalanced with setmaxnreg): warps 0-3 softmax,
+// warps 4-7 epilogue (O / l -> bf16 -> global, LSE) off the softmax warps' critical path,
+// warp 8 TMA producer, warp 9 MMA issuer / TMEM owner, warps 10-11 idle.
 // K and V tiles are double-buffered in shared memory and S in TMEM, so the next S = Q K^T is
 // issued while the softmax of the current tile runs.  The grid is persistent; two blocks
 // share an SM (256 TMEM columns each).  A small plan kernel turns the ragged layout into a
@@ -28,8 +29,8 @@ using namespace ptx;
 constexpr int kBM = 128;              // query rows per tile
 constexpr int kBN = 64;               // keys per tile
 constexpr int kHD = 128;              // head_dim
-constexpr int kSoftmaxWarps = 8;      // two threads per query row: each owns 32 of a tile's 64 keys
-constexpr int kTcThreads = (kSoftmaxWarps + 2) * 32;
+constexpr int kTmaWarp = 8, kMmaWarp = 9;
+constexpr int kTcThreads = 12 * 32;   // warps 0-3 softmax, 4-7 epilogue, 8 producer, 9 MMA issuer, 10-11 idle (warpgroup padding)
 constexpr int kQBytes = kBM * kHD * 2;     // 32 KB
 constexpr int kKVBytes = kBN * kHD * 2;    // 16 KB per stage
 constexpr int kTmemCols = 256;        // S/P double buffer: [0,64) [64,128)   O: [128,256)
@@ -186,12 +187,14 @@ struct Cursor {
 
 // S_FULL[st] (S = Q K^T of a tile complete) also tells the producer that K stage st is free;
 // O_DONE[st] (O += P V complete) also frees V stage st: one tcgen05.commit serves both waiters.
-// X_MAX[parity] / X_SUM: the two threads of a row exchange their half-row maximum (per
-// tile) and half-row sum (per item) through shared memory; mbarriers rather than bar.sync so
-// that these waits are bounded like all others.
+// L_READY: the softmax warps have published an item's row sums; O_FREE: the epilogue warps
+// have read the item's O out of tensor memory, so the next item's first O = P V may overwrite it.
 enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_V_FULL = BAR_K_FULL + 2, BAR_S_FULL = BAR_V_FULL + 2,
-       BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2, BAR_X_MAX = BAR_O_DONE + 2,
-       BAR_X_SUM = BAR_X_MAX + 2, BAR_DRAIN, BAR_COUNT };
+       BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2, BAR_L_READY = BAR_O_DONE + 2, BAR_O_FREE,
+       BAR_DRAIN, BAR_COUNT };
+
+template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_constant__ TcParams p)
 {
@@ -200,19 +203,20 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
     unsigned char *sQ = smem;                                   // 128 rows x 128 cols, two 64-col halves
     unsigned char *sK = smem + kQBytes;                         // [2 stages] 64 keys x 128 cols
     unsigned char *sV = sK + 2 * kKVBytes;                      // [2 stages]
-    unsigned char *sO = sV + 2 * kKVBytes;                      // [8 warps] 32 rows x 32 bytes, output staging
+    unsigned char *sO = sV + 2 * kKVBytes;                      // [4 warps] 32 rows x 64 bytes, output staging
     __shared__ uint64_t bars[BAR_COUNT];
     __shared__ uint32_t tmem_base_s;
-    __shared__ float x_max[2][2][kBM];                          // [tile parity][half][row]
-    __shared__ float x_sum[2][2][kBM];                          // [item parity][half][row]
+    __shared__ float x_l[2][kBM];                               // [item parity][row] row sums
+    __shared__ float x_m[2][kBM];                               // [item parity][row] reference maxima
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int i = 0; i < BAR_COUNT; ++i) mbar_init(&bars[i], (i >= BAR_P_FULL && i < BAR_P_FULL + 2) || (i >= BAR_X_MAX && i <= BAR_X_SUM) ? kSoftmaxWarps * 32 : 1);
+        for (int i = 0; i < BAR_COUNT; ++i)
+            mbar_init(&bars[i], (i == BAR_P_FULL || i == BAR_P_FULL + 1 || i == BAR_L_READY || i == BAR_O_FREE) ? 128 : 1);
         fence_mbar_init();
         prefetch_tmap(&p.mq); prefetch_tmap(&p.mk); prefetch_tmap(&p.mv);
     }
-    if (warp == kSoftmaxWarps + 1) { tmem_alloc(&tmem_base_s, kTmemCols); tmem_relinquish(); }
+    if (warp == kMmaWarp) { tmem_alloc(&tmem_base_s, kTmemCols); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -220,293 +224,313 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
     const uint32_t n_items = p.hdr->n_tiles * (uint32_t)p.n_heads;
     bool ok = true;
 
-    if (warp == kSoftmaxWarps) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            uint32_t nq = 0, nk[2] = {0, 0}, nv[2] = {0, 0};     // loads issued per "full" barrier
-            Cursor c;
-            for (c.init(p.tiles, n_items, p.n_heads); c.valid && ok && !p.stall_producer; c.next()) {
-                const int hk = c.h / p.kv_group;
-                if (c.j == 0) {
-                    if (!(ok = mbar_wait(&bars[BAR_Q_EMPTY], (c.item_no & 1) ^ 1))) break;
-                    mbar_expect_tx(&bars[BAR_Q_FULL], kQBytes);
-                    tma_load_2d(sQ, &p.mq, c.h * kHD, c.t.q_row, &bars[BAR_Q_FULL]);
-                    tma_load_2d(sQ + kQBytes / 2, &p.mq, c.h * kHD + 64, c.t.q_row, &bars[BAR_Q_FULL]);
-                    ++nq;
+    if (warp >= 8) {
+        reg_dealloc<40>();              // warps 8-11: producer, MMA issuer and two idle warps
+        if (warp == kTmaWarp) {
+            // -------------------------------------------------------------- TMA producer
+            if (lane == 0) {
+                uint32_t nq = 0, nk[2] = {0, 0}, nv[2] = {0, 0};     // loads issued per "full" barrier
+                Cursor c;
+                for (c.init(p.tiles, n_items, p.n_heads); c.valid && ok && !p.stall_producer; c.next()) {
+                    const int hk = c.h / p.kv_group;
+                    if (c.j == 0) {
+                        if (!(ok = mbar_wait(&bars[BAR_Q_EMPTY], (c.item_no & 1) ^ 1))) break;
+                        mbar_expect_tx(&bars[BAR_Q_FULL], kQBytes);
+                        tma_load_2d(sQ, &p.mq, c.h * kHD, c.t.q_row, &bars[BAR_Q_FULL]);
+                        tma_load_2d(sQ + kQBytes / 2, &p.mq, c.h * kHD + 64, c.t.q_row, &bars[BAR_Q_FULL]);
+                        ++nq;
+                    }
+                    const KvTile kt = c.kv();
+                    const int st = c.g & 1;
+                    const uint32_t ph = (c.g >> 1) & 1;
+                    if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], ph ^ 1))) break;       // K stage free
+                    mbar_expect_tx(&bars[BAR_K_FULL + st], kKVBytes);
+                    tma_load_2d(sK + st * kKVBytes, &p.mk, hk * kHD, kt.row0, &bars[BAR_K_FULL + st]);
+                    tma_load_2d(sK + st * kKVBytes + kKVBytes / 2, &p.mk, hk * kHD + 64, kt.row0, &bars[BAR_K_FULL + st]);
+                    ++nk[st];
+                    if (!(ok = mbar_wait(&bars[BAR_O_DONE + st], ph ^ 1))) break;       // V stage free
+                    mbar_expect_tx(&bars[BAR_V_FULL + st], kKVBytes);
+                    tma_load_2d(sV + st * kKVBytes, &p.mv, hk * kHD, kt.row0, &bars[BAR_V_FULL + st]);
+                    tma_load_2d(sV + st * kKVBytes + kKVBytes / 2, &p.mv, hk * kHD + 64, kt.row0, &bars[BAR_V_FULL + st]);
+                    ++nv[st];
                 }
-                const KvTile kt = c.kv();
-                const int st = c.g & 1;
-                const uint32_t ph = (c.g >> 1) & 1;
-                if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], ph ^ 1))) break;       // K stage free
-                mbar_expect_tx(&bars[BAR_K_FULL + st], kKVBytes);
-                tma_load_2d(sK + st * kKVBytes, &p.mk, hk * kHD, kt.row0, &bars[BAR_K_FULL + st]);
-                tma_load_2d(sK + st * kKVBytes + kKVBytes / 2, &p.mk, hk * kHD + 64, kt.row0, &bars[BAR_K_FULL + st]);
-                ++nk[st];
-                if (!(ok = mbar_wait(&bars[BAR_O_DONE + st], ph ^ 1))) break;       // V stage free
-                mbar_expect_tx(&bars[BAR_V_FULL + st], kKVBytes);
-                tma_load_2d(sV + st * kKVBytes, &p.mv, hk * kHD, kt.row0, &bars[BAR_V_FULL + st]);
-                tma_load_2d(sV + st * kKVBytes + kKVBytes / 2, &p.mv, hk * kHD + 64, kt.row0, &bars[BAR_V_FULL + st]);
-                ++nv[st];
-            }
-            if (!ok) {
-                // a wait ran out: before the block may exit, its own copies in flight must
-                // have landed (bounded waits on the phase of the last load of each buffer)
-                if (nq) mbar_wait(&bars[BAR_Q_FULL], (nq - 1) & 1);
-                for (int st = 0; st < 2; ++st) {
-                    if (nk[st]) mbar_wait(&bars[BAR_K_FULL + st], (nk[st] - 1) & 1);
-                    if (nv[st]) mbar_wait(&bars[BAR_V_FULL + st], (nv[st] - 1) & 1);
+                if (!ok) {
+                    // a wait ran out: before the block may exit, its own copies in flight must
+                    // have landed (bounded waits on the phase of the last load of each buffer)
+                    if (nq) mbar_wait(&bars[BAR_Q_FULL], (nq - 1) & 1);
+                    for (int st = 0; st < 2; ++st) {
+                        if (nk[st]) mbar_wait(&bars[BAR_K_FULL + st], (nk[st] - 1) & 1);
+                        if (nv[st]) mbar_wait(&bars[BAR_V_FULL + st], (nv[st] - 1) & 1);
+                    }
                 }
             }
-        }
-        __syncwarp();
-    } else if (warp == kSoftmaxWarps + 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            // Descriptor words are loop-invariant up to a small address offset: build them once.
-            // High word: stride-dimension offset 1024 B (8-row groups), descriptor version 1, 128B swizzle.
-            const uint32_t d_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-            const uint32_t q_lo = ((smem_u32(sQ) & 0x3ffffu) >> 4) | (1u << 16);
-            const uint32_t k_lo = ((smem_u32(sK) & 0x3ffffu) >> 4) | (1u << 16);
-            const uint32_t v_lo = ((smem_u32(sV) & 0x3ffffu) >> 4) | ((uint32_t)((kKVBytes / 2) >> 4) << 16);
-            const uint32_t id_o = idesc_bf16(kBM, kHD, 0, 1);
-            Cursor cs, cp;                      // cs: next S = Q K^T to issue; cp: next O += P V to issue
-            cs.init(p.tiles, n_items, p.n_heads);
-            cp.init(p.tiles, n_items, p.n_heads);
+        } else if (warp == kMmaWarp) {
+            // -------------------------------------------------------------- MMA issuer
+            if (lane == 0) {
+                // Descriptor words are loop-invariant up to a small address offset: build them once.
+                // High word: stride-dimension offset 1024 B (8-row groups), descriptor version 1, 128B swizzle.
+                const uint32_t d_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+                const uint32_t q_lo = ((smem_u32(sQ) & 0x3ffffu) >> 4) | (1u << 16);
+                const uint32_t k_lo = ((smem_u32(sK) & 0x3ffffu) >> 4) | (1u << 16);
+                const uint32_t v_lo = ((smem_u32(sV) & 0x3ffffu) >> 4) | ((uint32_t)((kKVBytes / 2) >> 4) << 16);
+                const uint32_t id_o = idesc_bf16(kBM, kHD, 0, 1);
+                Cursor cs, cp;                      // cs: next S = Q K^T to issue; cp: next O += P V to issue
+                cs.init(p.tiles, n_items, p.n_heads);
+                cp.init(p.tiles, n_items, p.n_heads);
 
-            while (cp.valid && ok) {
-                // S = Q K^T: the current tile's must be issued; the next tile's is issued one
-                // ahead of the softmax as soon as its operands have landed
-                while (cs.valid && (cs.g == cp.g ||
-                                    (cs.g == cp.g + 1 && (cs.j != 0 || mbar_test(&bars[BAR_Q_FULL], cs.item_no & 1)) &&
-                                     mbar_test(&bars[BAR_K_FULL + (cs.g & 1)], (cs.g >> 1) & 1)))) {
-                    const uint32_t st = cs.g & 1;
-                    if (cs.j == 0 && !(ok = mbar_wait(&bars[BAR_Q_FULL], cs.item_no & 1))) break;
-                    if (!(ok = mbar_wait(&bars[BAR_K_FULL + st], (cs.g >> 1) & 1))) break;
+                while (cp.valid && ok) {
+                    // S = Q K^T: the current tile's must be issued; the next tile's is issued one
+                    // ahead of the softmax as soon as its operands have landed
+                    while (cs.valid && (cs.g == cp.g ||
+                                        (cs.g == cp.g + 1 && (cs.j != 0 || mbar_test(&bars[BAR_Q_FULL], cs.item_no & 1)) &&
+                                         mbar_test(&bars[BAR_K_FULL + (cs.g & 1)], (cs.g >> 1) & 1)))) {
+                        const uint32_t st = cs.g & 1;
+                        if (cs.j == 0 && !(ok = mbar_wait(&bars[BAR_Q_FULL], cs.item_no & 1))) break;
+                        if (!(ok = mbar_wait(&bars[BAR_K_FULL + st], (cs.g >> 1) & 1))) break;
+                        tc_fence_after();
+                        const int n_mma = (cs.kv().n_valid + 15) & ~15;
+                        const uint32_t id_s = idesc_bf16(kBM, 0, 0, 0) | ((uint32_t)(n_mma >> 3) << 17);
+                        const uint32_t kb = k_lo + st * (kKVBytes >> 4);
+                        const uint32_t d = tb + st * kBN;
+#pragma unroll
+                        for (int kk = 0; kk < kHD / 16; ++kk)              // contraction over head_dim
+                            umma_ss_lh(d, q_lo + (kk >> 2) * (kQBytes >> 5) + (kk & 3) * 2,
+                                       kb + (kk >> 2) * (kKVBytes >> 5) + (kk & 3) * 2, d_hi, id_s, kk > 0 ? 1u : 0u);
+                        umma_commit(&bars[BAR_S_FULL + st]);
+                        if (cs.last_of_item()) umma_commit(&bars[BAR_Q_EMPTY]);
+                        cs.next();
+                    }
+                    if (!ok) break;
+                    const uint32_t st = cp.g & 1;
+                    const uint32_t ph = (cp.g >> 1) & 1;
+                    const int n_k = (cp.kv().n_valid + 15) >> 4;          // 16-key steps
+                    if (!(ok = mbar_wait(&bars[BAR_P_FULL + st], ph))) break;
+                    if (!(ok = mbar_wait(&bars[BAR_V_FULL + st], ph))) break;
+                    // the first O = P V of an item overwrites O: the previous item's must have been read out
+                    if (cp.j == 0 && cp.item_no > 0 && !(ok = mbar_wait(&bars[BAR_O_FREE], (cp.item_no - 1) & 1))) break;
                     tc_fence_after();
-                    const int n_mma = (cs.kv().n_valid + 15) & ~15;
-                    const uint32_t id_s = idesc_bf16(kBM, 0, 0, 0) | ((uint32_t)(n_mma >> 3) << 17);
-                    const uint32_t kb = k_lo + st * (kKVBytes >> 4);
-                    const uint32_t d = tb + st * kBN;
+                    const uint32_t vb = v_lo + st * (kKVBytes >> 4);
+                    const uint32_t pa = tb + st * kBN;
 #pragma unroll
-                    for (int kk = 0; kk < kHD / 16; ++kk)              // contraction over head_dim
-                        umma_ss_lh(d, q_lo + (kk >> 2) * (kQBytes >> 5) + (kk & 3) * 2,
-                                   kb + (kk >> 2) * (kKVBytes >> 5) + (kk & 3) * 2, d_hi, id_s, kk > 0 ? 1u : 0u);
-                    umma_commit(&bars[BAR_S_FULL + st]);
-                    if (cs.last_of_item()) umma_commit(&bars[BAR_Q_EMPTY]);
-                    cs.next();
+                    for (int kk = 0; kk < kBN / 16; ++kk)                 // contraction over keys
+                        if (kk < n_k)
+                            umma_ts_lh(tb + 128, pa + kk * 8, vb + kk * (2048 >> 4), d_hi, id_o, (cp.j > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(&bars[BAR_O_DONE + st]);
+                    cp.next();
                 }
-                if (!ok) break;
-                const uint32_t st = cp.g & 1;
-                const uint32_t ph = (cp.g >> 1) & 1;
-                const int n_k = (cp.kv().n_valid + 15) >> 4;          // 16-key steps
-                if (!(ok = mbar_wait(&bars[BAR_P_FULL + st], ph))) break;
-                if (!(ok = mbar_wait(&bars[BAR_V_FULL + st], ph))) break;
-                tc_fence_after();
-                const uint32_t vb = v_lo + st * (kKVBytes >> 4);
-                const uint32_t pa = tb + st * kBN;
-#pragma unroll
-                for (int kk = 0; kk < kBN / 16; ++kk)                 // contraction over keys
-                    if (kk < n_k)
-                        umma_ts_lh(tb + 128, pa + kk * 8, vb + kk * (2048 >> 4), d_hi, id_o, (cp.j > 0 || kk > 0) ? 1u : 0u);
-                umma_commit(&bars[BAR_O_DONE + st]);
-                cp.next();
-            }
-            if (!ok) {
-                // a wait ran out: let every MMA already issued finish (bounded) before the
-                // tensor memory they write is freed
-                umma_commit(&bars[BAR_DRAIN]);
-                mbar_wait(&bars[BAR_DRAIN], 0);
+                if (!ok) {
+                    // a wait ran out: let every MMA already issued finish (bounded) before the
+                    // tensor memory they write is freed
+                    umma_commit(&bars[BAR_DRAIN]);
+                    mbar_wait(&bars[BAR_DRAIN], 0);
+                }
             }
         }
         __syncwarp();
-    } else {
-        // ------------------------------------------------------------------ softmax + epilogue
-        // Thread (row, hf): TMEM lanes are reachable by warp % 4, so warps w and w + 4 share the
-        // same 32 rows; hf = warp / 4 picks keys [32 hf, 32 hf + 32) of every 64-key tile and
-        // output columns [64 hf, 64 hf + 64).
-        const int quad = warp & 3, hf = warp >> 2;
-        const int row = quad * 32 + lane;
-        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    } else if (warp < 4) {
+        // ------------------------------------------------------------------ softmax
+        // One thread per query row; a tile's 64 scores stay in registers (one TMEM read).
+        reg_alloc<120>();
+        const int row = warp * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
         const float sc = p.scale_log2e;
-        unsigned char *stage = sO + warp * 1024;
         Cursor c;
         c.init(p.tiles, n_items, p.n_heads);
-        float m_ref = -INFINITY, l = 0.f;          // reference maximum (log2 units), this thread's half of the row sum
-        // A finished item whose output is still in TMEM: its epilogue runs after the softmax of
-        // the next item's first tile, so the wait for its last O += P V is hidden behind work.
-        bool have_prev = false;
-        TcTile prev_t = {};
-        int prev_h = 0;
-        uint32_t prev_no = 0;
-        float prev_m = 0.f, prev_l = 1.f;
+        float m_ref = -INFINITY, l = 0.f;          // reference maximum (log2 units) and row sum
 
-        while ((c.valid || have_prev) && ok) {
+        while (c.valid && ok) {
             const int st = c.g & 1;
-            const bool first = c.valid && c.j == 0;
-            if (c.valid) {
-                const TcTile &t = c.t;
-                const KvTile kt = c.kv();
-                const uint32_t s_addr = tb + lane_addr + st * kBN + hf * 32;
-                const int n_mma = (kt.n_valid + 15) & ~15;
-                // keys of my 32 that this row / the warp's first and last rows may see
-                const int vis = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + row - kt.k_off + 1);
-                const int vis0 = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + quad * 32 - kt.k_off + 1);
-                const int vis31 = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + quad * 32 + 31 - kt.k_off + 1);
-                const int lim = vis - hf * 32;
-                // A warp whose 32 rows lie past the tile's last valid row does no arithmetic at all:
-                // its rows of P and O are never stored (it still takes part in every barrier).
-                const bool live_w = quad * 32 < t.n_rows;
-                const bool in_use = live_w && hf * 32 < n_mma;   // uniform: my part of P is read by O += P V and matters
-                const bool any_vis = live_w && vis31 - hf * 32 > 0;   // uniform: some row of the warp sees some key of mine
-                if (first) { m_ref = -INFINITY; l = 0.f; }
-                if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
-                tc_fence_after();
+            const bool first = c.j == 0;
+            const TcTile &t = c.t;
+            const KvTile kt = c.kv();
+            const uint32_t s_addr = tb + lane_addr + st * kBN;
+            const int n_mma = (kt.n_valid + 15) & ~15;
+            // keys this row / the warp's first and last rows may see
+            const int lim = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + row - kt.k_off + 1);
+            const int lim0 = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + warp * 32 - kt.k_off + 1);
+            const int lim31 = kt.k_off < 0 ? kt.n_valid : min(kt.n_valid, t.q_off + warp * 32 + 31 - kt.k_off + 1);
+            // A warp whose 32 rows lie past the tile's last valid row does no arithmetic at all:
+            // its rows of P and O are never stored (it still takes part in every barrier).
+            const bool live_w = warp * 32 < t.n_rows;
+            const bool use0 = live_w && lim31 > 0;               // uniform: keys [0,32) seen by some row
+            const bool use1 = live_w && lim31 > 32;              // uniform: keys [32,64) seen by some row
+            if (first) { m_ref = -INFINITY; l = 0.f; }
+            if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
+            tc_fence_after();
 
-                // My half of the row's scores stays in registers: one TMEM read per tile.
-                uint32_t r[32];
-                float hmax = -INFINITY;
-                if (any_vis) {
-                    tmem_ld32(s_addr, r);
-                    tmem_ld_wait();
-                    // keys past the row's limit (causal diagonal, ragged tail) -> -inf; skipped
-                    // when the whole warp sees all 32
-                    if (vis0 - hf * 32 < 32) {
+            uint32_t r0[32], r1[32];
+            if (use0) tmem_ld32(s_addr, r0);
+            if (use1) tmem_ld32(s_addr + 32, r1);
+            tmem_ld_wait();
+            // keys past the row's limit (causal diagonal, ragged tail) -> -inf; skipped when the
+            // whole warp sees everything it loaded
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            if (use0) {
+                if (lim0 < 32) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = (i < lim) ? r[i] : 0xff800000u;
-                    }
-                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                    for (int i = 0; i < 32; ++i) r0[i] = (i < lim) ? r0[i] : 0xff800000u;
+                }
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(r[i]));
-                    hmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(r0[i]));
+            }
+            if (use1) {
+                if (lim0 < 64) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r1[i] = (32 + i < lim) ? r1[i] : 0xff800000u;
                 }
-                // exchange the half-row maxima
-                x_max[st][hf][row] = hmax;
-                mbar_arrive(&bars[BAR_X_MAX + st]);
-                if (!(ok = mbar_wait(&bars[BAR_X_MAX + st], (c.g >> 1) & 1))) break;
-                const float m_tile = fmaxf(hmax, x_max[st][hf ^ 1][row]) * sc;
-                float alpha = 1.f;
-                bool grow = false;
-                if (first) {
-                    m_ref = m_tile;
-                } else if (m_tile > m_ref + kRescaleThreshold) {
-                    alpha = ex2(m_ref - m_tile);
-                    m_ref = m_tile;
-                    grow = true;
-                }
-                if (__any_sync(0xffffffffu, grow)) {     // rare: bring O and l to the new reference
-                    // needs the previous tile's O += P V complete; it is observed again below,
-                    // which returns at once (same phase)
-                    if (!(ok = mbar_wait(&bars[BAR_O_DONE + ((c.g - 1) & 1)], ((c.g - 1) >> 1) & 1))) break;
-                    tc_fence_after();
-                    l *= alpha;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(r1[i]));
+            }
+            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;
+            float alpha = 1.f;
+            bool grow = false;
+            if (first) {
+                m_ref = m_tile;
+            } else if (m_tile > m_ref + kRescaleThreshold) {
+                alpha = ex2(m_ref - m_tile);
+                m_ref = m_tile;
+                grow = true;
+            }
+            if (__any_sync(0xffffffffu, grow)) {     // rare: bring O and l to the new reference
+                // needs the previous tile's O += P V complete
+                if (!(ok = mbar_wait(&bars[BAR_O_DONE + ((c.g - 1) & 1)], ((c.g - 1) >> 1) & 1))) break;
+                tc_fence_after();
+                l *= alpha;
 #pragma unroll 1
-                    for (int cc = 0; cc < 2; ++cc) {
-                        uint32_t o[32];
-                        tmem_ld32(tb + lane_addr + 128 + hf * 64 + cc * 32, o);
-                        tmem_ld_wait();
+                for (int cc = 0; cc < kHD / 32; ++cc) {
+                    uint32_t o[32];
+                    tmem_ld32(tb + lane_addr + 128 + cc * 32, o);
+                    tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st32(tb + lane_addr + 128 + hf * 64 + cc * 32, o);
-                    }
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st32(tb + lane_addr + 128 + cc * 32, o);
                 }
-                if (in_use) {
-                    const uint32_t p_addr = tb + lane_addr + st * kBN + hf * 16;
-                    if (any_vis) {
-                        // masked scores are -inf, so exp2 gives exactly 0 for them
-                        const float nm = -m_ref;
-                        float rs[4] = {0.f, 0.f, 0.f, 0.f};
+            }
+            if (live_w) {
+                // masked scores are -inf, so exp2 gives exactly 0 for them
+                const float nm = -m_ref;
+                float rs[4] = {0.f, 0.f, 0.f, 0.f};
+                if (use0) {
 #pragma unroll
-                        for (int q8 = 0; q8 < 2; ++q8) {          // 16 keys -> 8 packed pairs per store
+                    for (int q8 = 0; q8 < 2; ++q8) {              // 16 keys -> 8 packed pairs per store
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int i = 0; i < 16; i += 2) {
+                            const float p0 = ex2(fmaf(__uint_as_float(r0[q8 * 16 + i]), sc, nm));
+                            const float p1 = ex2(fmaf(__uint_as_float(r0[q8 * 16 + i + 1]), sc, nm));
+                            rs[(i >> 1) & 3] += p0 + p1;
+                            pk[i >> 1] = pack_bf16x2(p0, p1);
+                        }
+                        tmem_st8(s_addr + q8 * 8, pk);
+                    }
+                } else {
+                    uint32_t z[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) z[i] = 0u;
+                    tmem_st8(s_addr, z);
+                    tmem_st8(s_addr + 8, z);
+                }
+                if (n_mma > 32) {
+                    if (use1) {
+#pragma unroll
+                        for (int q8 = 0; q8 < 2; ++q8) {
                             uint32_t pk[8];
 #pragma unroll
                             for (int i = 0; i < 16; i += 2) {
-                                const float p0 = ex2(fmaf(__uint_as_float(r[q8 * 16 + i]), sc, nm));
-                                const float p1 = ex2(fmaf(__uint_as_float(r[q8 * 16 + i + 1]), sc, nm));
+                                const float p0 = ex2(fmaf(__uint_as_float(r1[q8 * 16 + i]), sc, nm));
+                                const float p1 = ex2(fmaf(__uint_as_float(r1[q8 * 16 + i + 1]), sc, nm));
                                 rs[(i >> 1) & 3] += p0 + p1;
                                 pk[i >> 1] = pack_bf16x2(p0, p1);
                             }
-                            tmem_st8(p_addr + q8 * 8, pk);
+                            tmem_st8(s_addr + 16 + q8 * 8, pk);
                         }
-                        l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
                     } else {
                         uint32_t z[8];
 #pragma unroll
                         for (int i = 0; i < 8; ++i) z[i] = 0u;
-                        tmem_st8(p_addr, z);
-                        tmem_st8(p_addr + 8, z);
+                        tmem_st8(s_addr + 16, z);
+                        tmem_st8(s_addr + 24, z);
                     }
                 }
+                l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
             }
-            // Every completion of O += P V is observed exactly once per stage, in order (tile
-            // g - 1 here), so the barrier parity stays unambiguous.
-            if (c.g > 0 && !(ok = mbar_wait(&bars[BAR_O_DONE + ((c.g - 1) & 1)], ((c.g - 1) >> 1) & 1))) break;
-
-            if (have_prev && (first || !c.valid)) {
-                // ---- epilogue of the previous item: O / l -> bf16 -> global (my 64 columns)
-                tc_fence_after();
-                const int xp = prev_no & 1;
-                x_sum[xp][hf][row] = prev_l;
-                mbar_arrive(&bars[BAR_X_SUM]);
-                if (!(ok = mbar_wait(&bars[BAR_X_SUM], xp))) break;
-                const float l_row = prev_l + x_sum[xp][hf ^ 1][row];
-                const float inv = 1.f / l_row;
-                if (quad * 32 < prev_t.n_rows) {
-                unsigned char *dst = reinterpret_cast<unsigned char *>(p.out) +
-                                     ((int64_t)prev_t.q_row * p.n_heads + prev_h) * (kHD * 2) + hf * 128;
-                const int64_t row_pitch = (int64_t)p.n_heads * kHD * 2;
-#pragma unroll 1
-                for (int cc = 0; cc < 2; ++cc) {
-                    uint32_t ro[32];
-                    tmem_ld32(tb + lane_addr + 128 + hf * 64 + cc * 32, ro);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int sub = 0; sub < 2; ++sub) {      // 16 output columns (32 bytes per row) per round
-                        // thread = row -> shared staging (xor-swizzled 16-byte pieces) -> each store
-                        // instruction writes 16 rows x 32 contiguous bytes
-#pragma unroll
-                        for (int q2 = 0; q2 < 2; ++q2) {
-                            const int e = sub * 16 + q2 * 8;
-                            uint4 w;
-                            w.x = pack_bf16x2(__uint_as_float(ro[e + 0]) * inv, __uint_as_float(ro[e + 1]) * inv);
-                            w.y = pack_bf16x2(__uint_as_float(ro[e + 2]) * inv, __uint_as_float(ro[e + 3]) * inv);
-                            w.z = pack_bf16x2(__uint_as_float(ro[e + 4]) * inv, __uint_as_float(ro[e + 5]) * inv);
-                            w.w = pack_bf16x2(__uint_as_float(ro[e + 6]) * inv, __uint_as_float(ro[e + 7]) * inv);
-                            *reinterpret_cast<uint4 *>(stage + lane * 32 + ((q2 ^ ((lane >> 2) & 1)) << 4)) = w;
-                        }
-                        __syncwarp();
-#pragma unroll
-                        for (int i = 0; i < 2; ++i) {
-                            const int rr = (lane >> 1) + 16 * i, piece = lane & 1;
-                            const uint4 w = *reinterpret_cast<const uint4 *>(stage + rr * 32 + ((piece ^ ((rr >> 2) & 1)) << 4));
-                            if (quad * 32 + rr < prev_t.n_rows)
-                                *reinterpret_cast<uint4 *>(dst + (int64_t)(quad * 32 + rr) * row_pitch + (cc * 2 + sub) * 32 + piece * 16) = w;
-                        }
-                        __syncwarp();
-                    }
-                }
-                if (hf == 0 && row < prev_t.n_rows && p.lse)
-                    p.lse[(int64_t)prev_h * p.total_tokens + prev_t.q_row + row] = (prev_m + log2f(l_row)) * kLn2T;
-                }
-                have_prev = false;
-            }
-            if (!c.valid) break;
-
-            // P of this tile is in TMEM (and O of the previous item has been read out): release
-            // the tile to the MMA issuer
+            // P of this tile is in TMEM: release the tile to the MMA issuer
             tmem_st_wait();
             tc_fence_before();
             mbar_arrive(&bars[BAR_P_FULL + st]);
-            if (c.last_of_item()) {
-                have_prev = true; prev_t = c.t; prev_h = c.h; prev_m = m_ref; prev_l = l; prev_no = c.item_no;
+            if (c.last_of_item()) {                 // hand the item's row statistics to the epilogue warps
+                x_l[c.item_no & 1][row] = l;
+                x_m[c.item_no & 1][row] = m_ref;
+                mbar_arrive(&bars[BAR_L_READY]);
             }
             c.next();
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 4-7)
+        // O / l -> bf16 -> global and the log-sum-exp, off the softmax warps' critical path.
+        const int quad = warp - 4;
+        const int row = quad * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        unsigned char *stage = sO + quad * 2048;
+        const int64_t row_pitch = (int64_t)p.n_heads * kHD * 2;
+        uint32_t g_end = 0, item_no = 0;
+        for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++item_no) {
+            const uint32_t ti = it / (uint32_t)p.n_heads;
+            const TcTile t = p.tiles[ti];
+            const int h = (int)(it - ti * (uint32_t)p.n_heads);
+            g_end += (t.pre_len + kBN - 1) / kBN + (t.q_off + t.n_rows + kBN - 1) / kBN;
+            const uint32_t g_last = g_end - 1;
+            const int xp = item_no & 1;
+            if (!(ok = mbar_wait(&bars[BAR_L_READY], xp))) break;
+            const float l_row = x_l[xp][row], m_row = x_m[xp][row];
+            if (!(ok = mbar_wait(&bars[BAR_O_DONE + (g_last & 1)], (g_last >> 1) & 1))) break;   // last O += P V
+            tc_fence_after();
+            const float inv = 1.f / l_row;
+            unsigned char *dst = reinterpret_cast<unsigned char *>(p.out) + ((int64_t)t.q_row * p.n_heads + h) * (kHD * 2);
+            const bool live_w = quad * 32 < t.n_rows;
+#pragma unroll 1
+            for (int cc = 0; cc < kHD / 32; ++cc) {
+                uint32_t ro[32];
+                if (live_w) {
+                    tmem_ld32(tb + lane_addr + 128 + cc * 32, ro);
+                    tmem_ld_wait();
+                }
+                if (cc == kHD / 32 - 1) {              // O is in registers: the accumulator may be overwritten
+                    tc_fence_before();
+                    mbar_arrive(&bars[BAR_O_FREE]);
+                }
+                if (live_w) {
+                    // thread = row -> shared staging (xor-swizzled 16-byte pieces) -> each store
+                    // instruction writes 8 rows x 64 contiguous bytes
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(ro[q4 * 8 + 0]) * inv, __uint_as_float(ro[q4 * 8 + 1]) * inv);
+                        w.y = pack_bf16x2(__uint_as_float(ro[q4 * 8 + 2]) * inv, __uint_as_float(ro[q4 * 8 + 3]) * inv);
+                        w.z = pack_bf16x2(__uint_as_float(ro[q4 * 8 + 4]) * inv, __uint_as_float(ro[q4 * 8 + 5]) * inv);
+                        w.w = pack_bf16x2(__uint_as_float(ro[q4 * 8 + 6]) * inv, __uint_as_float(ro[q4 * 8 + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(stage + lane * 64 + ((q4 ^ ((lane >> 1) & 3)) << 4)) = w;
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int rr = (lane >> 2) + 8 * i, piece = lane & 3;
+                        const uint4 w = *reinterpret_cast<const uint4 *>(stage + rr * 64 + ((piece ^ ((rr >> 1) & 3)) << 4));
+                        if (quad * 32 + rr < t.n_rows)
+                            *reinterpret_cast<uint4 *>(dst + (int64_t)(quad * 32 + rr) * row_pitch + cc * 64 + piece * 16) = w;
+                    }
+                    __syncwarp();
+                }
+            }
+            if (row < t.n_rows && p.lse)
+                p.lse[(int64_t)h * p.total_tokens + t.q_row + row] = (m_row + log2f(l_row)) * kLn2T;
         }
     }
 
     if (!ok && lane == 0) atomicExch(p.status, (uint32_t)STATUS_TIMEOUT);
     tc_fence_before();
     __syncthreads();
-    if (warp == kSoftmaxWarps + 1) tmem_dealloc(tb, kTmemCols);
+    if (warp == kMmaWarp) tmem_dealloc(tb, kTmemCols);
 }
 
 // ---- host side ---------------------------------------------------------------------------
@@ -584,7 +608,7 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
     const int64_t items = max_tiles(lay->n_prompts, lay->n_paths, lay->max_pre_len, lay->max_path_len) * n_heads;
     if (items == 0) return SP_OK;
     const int grid = (int)std::min<int64_t>(items, 2 * kNumSMs);
-    const int smem = kQBytes + 4 * kKVBytes + kSoftmaxWarps * 1024 + 1024;
+    const int smem = kQBytes + 4 * kKVBytes + 4 * 2048 + 1024;
     SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     prefill_tc_kernel<<<grid, kTcThreads, smem, st>>>(p);
     SP_CUDA(cudaGetLastError());
