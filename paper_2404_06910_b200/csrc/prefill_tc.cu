@@ -236,8 +236,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     if (c.j == 0) {
                         if (!(ok = mbar_wait(&bars[BAR_Q_EMPTY], (c.item_no & 1) ^ 1))) break;
                         mbar_expect_tx(&bars[BAR_Q_FULL], kQBytes);
-                        tma_load_2d(sQ, &p.mq, c.h * kHD, c.t.q_row, &bars[BAR_Q_FULL]);
-                        tma_load_2d(sQ + kQBytes / 2, &p.mq, c.h * kHD + 64, c.t.q_row, &bars[BAR_Q_FULL]);
+                        tma_load_3d(sQ, &p.mq, 0, c.t.q_row, c.h * 2, &bars[BAR_Q_FULL]);
                         ++nq;
                     }
                     const KvTile kt = c.kv();
@@ -245,13 +244,11 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     const uint32_t ph = (c.g >> 1) & 1;
                     if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], ph ^ 1))) break;       // K stage free
                     mbar_expect_tx(&bars[BAR_K_FULL + st], kKVBytes);
-                    tma_load_2d(sK + st * kKVBytes, &p.mk, hk * kHD, kt.row0, &bars[BAR_K_FULL + st]);
-                    tma_load_2d(sK + st * kKVBytes + kKVBytes / 2, &p.mk, hk * kHD + 64, kt.row0, &bars[BAR_K_FULL + st]);
+                    tma_load_3d(sK + st * kKVBytes, &p.mk, 0, kt.row0, hk * 2, &bars[BAR_K_FULL + st]);
                     ++nk[st];
                     if (!(ok = mbar_wait(&bars[BAR_O_DONE + st], ph ^ 1))) break;       // V stage free
                     mbar_expect_tx(&bars[BAR_V_FULL + st], kKVBytes);
-                    tma_load_2d(sV + st * kKVBytes, &p.mv, hk * kHD, kt.row0, &bars[BAR_V_FULL + st]);
-                    tma_load_2d(sV + st * kKVBytes + kKVBytes / 2, &p.mv, hk * kHD + 64, kt.row0, &bars[BAR_V_FULL + st]);
+                    tma_load_3d(sV + st * kKVBytes, &p.mv, 0, kt.row0, hk * 2, &bars[BAR_V_FULL + st]);
                     ++nv[st];
                 }
                 if (!ok) {
@@ -540,12 +537,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 static int encode_rows_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int64_t rows, int64_t cols, int box_rows)
 {
-    // [rows, cols] bf16 row-major; box = box_rows x 64 columns (128 bytes), 128-byte swizzle
-    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+    // [rows, cols] bf16 row-major seen as 3-D (64 columns, rows, cols / 64): one box = box_rows x
+    // 128 columns of one head, delivered as two 128-byte-swizzled halves [half][row][64 columns],
+    // which is the layout the MMA descriptors expect -- one TMA instruction per tile.
+    cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
+    cuuint64_t strides[2] = {(cuuint64_t)cols * 2, 128};
+    cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     SP_REQUIRE(r == CUDA_SUCCESS, SP_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
