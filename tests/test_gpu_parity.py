@@ -112,6 +112,14 @@ def test_prefill_ragged_edges(dtype, D):
     _check_prefill(lay, 4, 2, D, dtype, 100, std=1.0)
 
 
+@pytest.mark.parametrize("dtype,D", [("f32", 64), ("bf16", 128)])
+def test_prefill_fewer_rows_than_one_tile(dtype, D):
+    """Whole problems smaller than a single tile (the tensor is shorter than a TMA box)."""
+    for pre, docs, qrys in (([3], [[5]], [[2]]), ([0], [[0]], [[1]]), ([1, 2], [[1], [0, 3]], [[1], [1, 1]])):
+        lay = build_layout(pre, docs, qrys)
+        _check_prefill(lay, 2, 2, D, dtype, 900 + lay.total_tokens)
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_prefill_peaky_scores_and_planted_keys(dtype):
     """Unscaled N(0,1) q.k (sharp softmax) and one dominant key per row: masking or
