@@ -143,9 +143,18 @@ struct KvTile {
 // Walks the block's work: items (query tile, head) in a grid-stride order, and inside an
 // item its key tiles.  g counts key tiles since the block started: it selects the ring
 // stage (g & 1) and the barrier parity ((g >> 1) & 1) of every double-buffered resource.
+// Item number -> (query tile, head): heads vary fastest, so blocks running side by side read
+// neighbouring 256-byte head slices of the same token rows.
+__device__ __forceinline__ void item_decode(uint32_t it, uint32_t n_heads, uint32_t n_tiles, uint32_t &ti, int &h)
+{
+    (void)n_tiles;
+    ti = it / n_heads;
+    h = (int)(it - ti * n_heads);
+}
+
 struct Cursor {
     const TcTile *tiles;
-    uint32_t it, n_items, stride, g, item_no;
+    uint32_t it, n_items, n_tiles, stride, g, item_no;
     int n_heads, h, j, n_kv, n_pre;
     TcTile t;
     bool valid;
@@ -153,9 +162,9 @@ struct Cursor {
     {
         valid = it < n_items;
         if (valid) {
-            const uint32_t ti = it / (uint32_t)n_heads;
+            uint32_t ti;
+            item_decode(it, (uint32_t)n_heads, n_tiles, ti, h);
             t = tiles[ti];
-            h = (int)(it - ti * (uint32_t)n_heads);
             n_pre = (t.pre_len + kBN - 1) / kBN;
             n_kv = n_pre + (t.q_off + t.n_rows + kBN - 1) / kBN;
             j = 0;
@@ -174,7 +183,7 @@ struct Cursor {
     }
     __device__ __forceinline__ void init(const TcTile *tl, uint32_t n, int heads)
     {
-        tiles = tl; n_items = n; n_heads = heads; it = blockIdx.x; stride = gridDim.x; g = 0; item_no = 0;
+        tiles = tl; n_items = n; n_heads = heads; n_tiles = n / (uint32_t)heads; it = blockIdx.x; stride = gridDim.x; g = 0; item_no = 0;
         load();
     }
     __device__ __forceinline__ void next()
@@ -187,11 +196,16 @@ struct Cursor {
 
 // S_FULL[st] (S = Q K^T of a tile complete) also tells the producer that K stage st is free;
 // O_DONE[st] (O += P V complete) also frees V stage st: one tcgen05.commit serves both waiters.
-// L_READY: the softmax warps have published an item's row sums; O_FREE: the epilogue warps
-// have read the item's O out of tensor memory, so the next item's first O = P V may overwrite it.
+// L_READY[item parity]: the softmax warps have published an item's row sums; X_FREE[item parity]:
+// the epilogue warps have read them, so the slot may be rewritten two items later.  Both are
+// per-parity pairs because warps whose rows are masked out of a tile finish it almost at once:
+// with a single barrier their arrivals for the next one-tile item could complete the phase of
+// the current item before the warp on the diagonal has published its rows.
+// O_FREE: the epilogue warps have read the item's O out of tensor memory, so the next item's
+// first O = P V may overwrite it.
 enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_V_FULL = BAR_K_FULL + 2, BAR_S_FULL = BAR_V_FULL + 2,
-       BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2, BAR_L_READY = BAR_O_DONE + 2, BAR_O_FREE,
-       BAR_DRAIN, BAR_COUNT };
+       BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2, BAR_L_READY = BAR_O_DONE + 2,
+       BAR_X_FREE = BAR_L_READY + 2, BAR_O_FREE = BAR_X_FREE + 2, BAR_DRAIN, BAR_COUNT };
 
 template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
@@ -212,7 +226,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int i = 0; i < BAR_COUNT; ++i)
-            mbar_init(&bars[i], (i == BAR_P_FULL || i == BAR_P_FULL + 1 || i == BAR_L_READY || i == BAR_O_FREE) ? 128 : 1);
+            mbar_init(&bars[i], ((i >= BAR_P_FULL && i < BAR_P_FULL + 2) || (i >= BAR_L_READY && i <= BAR_O_FREE)) ? 128 : 1);
         fence_mbar_init();
         prefetch_tmap(&p.mq); prefetch_tmap(&p.mk); prefetch_tmap(&p.mv);
     }
@@ -456,9 +470,12 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             tc_fence_before();
             mbar_arrive(&bars[BAR_P_FULL + st]);
             if (c.last_of_item()) {                 // hand the item's row statistics to the epilogue warps
-                x_l[c.item_no & 1][row] = l;
-                x_m[c.item_no & 1][row] = m_ref;
-                mbar_arrive(&bars[BAR_L_READY]);
+                const uint32_t xp = c.item_no & 1;
+                // the slot was last used two items ago: the epilogue must have read it
+                if (c.item_no >= 2 && !(ok = mbar_wait(&bars[BAR_X_FREE + xp], ((c.item_no >> 1) - 1) & 1))) break;
+                x_l[xp][row] = l;
+                x_m[xp][row] = m_ref;
+                mbar_arrive(&bars[BAR_L_READY + xp]);
             }
             c.next();
         }
@@ -472,14 +489,16 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
         const int64_t row_pitch = (int64_t)p.n_heads * kHD * 2;
         uint32_t g_end = 0, item_no = 0;
         for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++item_no) {
-            const uint32_t ti = it / (uint32_t)p.n_heads;
+            uint32_t ti;
+            int h;
+            item_decode(it, (uint32_t)p.n_heads, p.hdr->n_tiles, ti, h);
             const TcTile t = p.tiles[ti];
-            const int h = (int)(it - ti * (uint32_t)p.n_heads);
             g_end += (t.pre_len + kBN - 1) / kBN + (t.q_off + t.n_rows + kBN - 1) / kBN;
             const uint32_t g_last = g_end - 1;
             const int xp = item_no & 1;
-            if (!(ok = mbar_wait(&bars[BAR_L_READY], xp))) break;
+            if (!(ok = mbar_wait(&bars[BAR_L_READY + xp], (item_no >> 1) & 1))) break;
             const float l_row = x_l[xp][row], m_row = x_m[xp][row];
+            mbar_arrive(&bars[BAR_X_FREE + xp]);
             if (!(ok = mbar_wait(&bars[BAR_O_DONE + (g_last & 1)], (g_last >> 1) & 1))) break;   // last O += P V
             tc_fence_after();
             const float inv = 1.f / l_row;

@@ -74,9 +74,11 @@ def _prefill_gpu(q, k, v, lay, scale, rows=sp.SP_ROWS_ALL, poison=True):
     return f32(out), lse.cpu().numpy()
 
 
-def _check_prefill(lay, H, Hkv, D, dtype, seed, std=1.0, scale=None):
+def _check_prefill(lay, H, Hkv, D, dtype, seed, std=1.0, scale=None, q_row_gain=None):
     T = lay.total_tokens
     q = _randn((T, H, D), dtype, seed, std)
+    if q_row_gain is not None:
+        q = (q.float() * torch.from_numpy(q_row_gain).float()[:, None, None]).to(q.dtype)
     k = _randn((T, Hkv, D), dtype, seed + 1, std)
     v = _randn((T, Hkv, D), dtype, seed + 2)
     scale = 1 / math.sqrt(D) if scale is None else scale
@@ -118,6 +120,24 @@ def test_prefill_fewer_rows_than_one_tile(dtype, D):
     for pre, docs, qrys in (([3], [[5]], [[2]]), ([0], [[0]], [[1]]), ([1, 2], [[1], [0, 3]], [[1], [1, 1]])):
         lay = build_layout(pre, docs, qrys)
         _check_prefill(lay, 2, 2, D, dtype, 900 + lay.total_tokens)
+
+
+def test_prefill_one_tile_items_follow_long_items():
+    """Work items with a single key tile (no preamble, a path shorter than one tile) right after
+    items with three key tiles in the same persistent block: warps whose rows are masked out of
+    the long item's last tile run ahead into the short item, which must not disturb the hand-off
+    of the long item's row sums.  With 2 heads a block's next item is 148 tiles further on."""
+    docs, qrys = [], []
+    for _ in range(3):
+        docs += [184] * 74 + [12] * 148          # 74 paths of 192 rows (2 tiles each), 148 of 20 rows
+        qrys += [8] * 74 + [8] * 148
+    lay = build_layout([0], [docs], [qrys])
+    # the middle third's queries are 6x larger, so its row sums and maxima differ widely from
+    # those of the items that used the same hand-off slot before and after
+    gain = np.ones(lay.total_tokens, dtype=np.float32)
+    gain[lay.total_tokens // 3: 2 * lay.total_tokens // 3] = 6.0
+    for rep in range(3):
+        _check_prefill(lay, 2, 2, 128, "bf16", 4242 + rep, q_row_gain=gain)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
