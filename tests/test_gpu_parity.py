@@ -183,9 +183,31 @@ def test_prefill_is_deterministic():
     lay = draw_lengths(cfg)
     q, k, v = draw_qkv(cfg, lay)
     a, la = _prefill_gpu(q, k, v, lay, 0.0884)
-    b, lb = _prefill_gpu(q, k, v, lay, 0.0884)
-    np.testing.assert_array_equal(a, b)
-    np.testing.assert_array_equal(la, lb)
+    for _ in range(5):
+        b, lb = _prefill_gpu(q, k, v, lay, 0.0884)
+        np.testing.assert_array_equal(a, b)
+        np.testing.assert_array_equal(la, lb)
+
+
+@pytest.mark.parametrize("case", ["mixed", "tiny_items", "preamble_only"])
+def test_prefill_random_ragged_layouts(case):
+    """Random segment lengths (empty documents and preambles included), grouped-query heads,
+    items of every size next to each other in the persistent blocks' work lists."""
+    rng = np.random.default_rng(3)
+    if case == "mixed":
+        lay = build_layout(list(rng.integers(0, 70, 4)), [list(rng.integers(0, 300, 30)) for _ in range(4)],
+                           [list(rng.integers(1, 40, 30)) for _ in range(4)])
+        H, Hkv = 8, 2
+    elif case == "tiny_items":
+        lay = build_layout([0] * 4, [list(rng.integers(0, 30, 200)) for _ in range(4)],
+                           [list(rng.integers(1, 8, 200)) for _ in range(4)])
+        H, Hkv = 4, 4
+    else:
+        lay = build_layout([700, 1, 129], [[], [], []], [[], [], []])
+        H, Hkv = 4, 1
+    gain = np.ones(lay.total_tokens, dtype=np.float32)
+    gain[lay.total_tokens // 3: 2 * lay.total_tokens // 3] = 5.0
+    _check_prefill(lay, H, Hkv, 128, "bf16", 77, q_row_gain=gain)
 
 
 # ------------------------------------------------------------------------- path scores
