@@ -59,8 +59,14 @@ struct TcHeader {                     // start of the workspace
     uint32_t n_tiles;
 };
 
+// Tiles with few valid rows are fetched through tensor maps with shorter boxes (32 or 64 rows
+// instead of 128 / 64), so that ragged tails and query-only tiles do not pull in rows nobody
+// needs.  A box lands as two swizzled halves of box_rows x 128 bytes each.
+__device__ __host__ __forceinline__ int q_box_sel(int n_rows) { return n_rows <= 32 ? 0 : (n_rows <= 64 ? 1 : 2); }
+__device__ __host__ __forceinline__ int kv_box_sel(int n_valid) { return n_valid <= 32 ? 0 : 1; }
+
 struct TcParams {
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mq[3], mk[2], mv[2];  // box rows: Q 32 / 64 / 128, K and V 32 / 64
     const TcHeader *hdr;
     const TcTile *tiles;
     uint32_t *status;
@@ -228,7 +234,8 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
         for (int i = 0; i < BAR_COUNT; ++i)
             mbar_init(&bars[i], ((i >= BAR_P_FULL && i < BAR_P_FULL + 2) || (i >= BAR_L_READY && i <= BAR_O_FREE)) ? 128 : 1);
         fence_mbar_init();
-        prefetch_tmap(&p.mq); prefetch_tmap(&p.mk); prefetch_tmap(&p.mv);
+        for (int i = 0; i < 3; ++i) prefetch_tmap(&p.mq[i]);
+        for (int i = 0; i < 2; ++i) { prefetch_tmap(&p.mk[i]); prefetch_tmap(&p.mv[i]); }
     }
     if (warp == kMmaWarp) { tmem_alloc(&tmem_base_s, kTmemCols); tmem_relinquish(); }
     tc_fence_before();
@@ -249,20 +256,22 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     const int hk = c.h / p.kv_group;
                     if (c.j == 0) {
                         if (!(ok = mbar_wait(&bars[BAR_Q_EMPTY], (c.item_no & 1) ^ 1))) break;
-                        mbar_expect_tx(&bars[BAR_Q_FULL], kQBytes);
-                        tma_load_3d(sQ, &p.mq, 0, c.t.q_row, c.h * 2, &bars[BAR_Q_FULL]);
+                        const int qs = q_box_sel(c.t.n_rows);
+                        mbar_expect_tx(&bars[BAR_Q_FULL], (32u << qs) * (kHD * 2));
+                        tma_load_3d(sQ, &p.mq[qs], 0, c.t.q_row, c.h * 2, &bars[BAR_Q_FULL]);
                         ++nq;
                     }
                     const KvTile kt = c.kv();
                     const int st = c.g & 1;
                     const uint32_t ph = (c.g >> 1) & 1;
                     if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], ph ^ 1))) break;       // K stage free
-                    mbar_expect_tx(&bars[BAR_K_FULL + st], kKVBytes);
-                    tma_load_3d(sK + st * kKVBytes, &p.mk, 0, kt.row0, hk * 2, &bars[BAR_K_FULL + st]);
+                    const int ks = kv_box_sel(kt.n_valid);
+                    mbar_expect_tx(&bars[BAR_K_FULL + st], (32u << ks) * (kHD * 2));
+                    tma_load_3d(sK + st * kKVBytes, &p.mk[ks], 0, kt.row0, hk * 2, &bars[BAR_K_FULL + st]);
                     ++nk[st];
                     if (!(ok = mbar_wait(&bars[BAR_O_DONE + st], ph ^ 1))) break;       // V stage free
-                    mbar_expect_tx(&bars[BAR_V_FULL + st], kKVBytes);
-                    tma_load_3d(sV + st * kKVBytes, &p.mv, 0, kt.row0, hk * 2, &bars[BAR_V_FULL + st]);
+                    mbar_expect_tx(&bars[BAR_V_FULL + st], (32u << ks) * (kHD * 2));
+                    tma_load_3d(sV + st * kKVBytes, &p.mv[ks], 0, kt.row0, hk * 2, &bars[BAR_V_FULL + st]);
                     ++nv[st];
                 }
                 if (!ok) {
@@ -283,7 +292,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 const uint32_t d_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
                 const uint32_t q_lo = ((smem_u32(sQ) & 0x3ffffu) >> 4) | (1u << 16);
                 const uint32_t k_lo = ((smem_u32(sK) & 0x3ffffu) >> 4) | (1u << 16);
-                const uint32_t v_lo = ((smem_u32(sV) & 0x3ffffu) >> 4) | ((uint32_t)((kKVBytes / 2) >> 4) << 16);
+                const uint32_t v_lo = (smem_u32(sV) & 0x3ffffu) >> 4;     // leading-dimension offset (half stride) added per tile
                 const uint32_t id_o = idesc_bf16(kBM, kHD, 0, 1);
                 Cursor cs, cp;                      // cs: next S = Q K^T to issue; cp: next O += P V to issue
                 cs.init(p.tiles, n_items, p.n_heads);
@@ -299,14 +308,18 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                         if (cs.j == 0 && !(ok = mbar_wait(&bars[BAR_Q_FULL], cs.item_no & 1))) break;
                         if (!(ok = mbar_wait(&bars[BAR_K_FULL + st], (cs.g >> 1) & 1))) break;
                         tc_fence_after();
-                        const int n_mma = (cs.kv().n_valid + 15) & ~15;
+                        const int n_valid = cs.kv().n_valid;
+                        const int n_mma = (n_valid + 15) & ~15;
                         const uint32_t id_s = idesc_bf16(kBM, 0, 0, 0) | ((uint32_t)(n_mma >> 3) << 17);
                         const uint32_t kb = k_lo + st * (kKVBytes >> 4);
                         const uint32_t d = tb + st * kBN;
+                        // second 64-column half of a box: box_rows x 128 bytes further on (in 16-byte units)
+                        const uint32_t q_half = (32u << q_box_sel(cs.t.n_rows)) * 8u;
+                        const uint32_t k_half = (32u << kv_box_sel(n_valid)) * 8u;
 #pragma unroll
                         for (int kk = 0; kk < kHD / 16; ++kk)              // contraction over head_dim
-                            umma_ss_lh(d, q_lo + (kk >> 2) * (kQBytes >> 5) + (kk & 3) * 2,
-                                       kb + (kk >> 2) * (kKVBytes >> 5) + (kk & 3) * 2, d_hi, id_s, kk > 0 ? 1u : 0u);
+                            umma_ss_lh(d, q_lo + (kk >> 2) * q_half + (kk & 3) * 2,
+                                       kb + (kk >> 2) * k_half + (kk & 3) * 2, d_hi, id_s, kk > 0 ? 1u : 0u);
                         umma_commit(&bars[BAR_S_FULL + st]);
                         if (cs.last_of_item()) umma_commit(&bars[BAR_Q_EMPTY]);
                         cs.next();
@@ -314,13 +327,14 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     if (!ok) break;
                     const uint32_t st = cp.g & 1;
                     const uint32_t ph = (cp.g >> 1) & 1;
-                    const int n_k = (cp.kv().n_valid + 15) >> 4;          // 16-key steps
+                    const int pv_valid = cp.kv().n_valid;
+                    const int n_k = (pv_valid + 15) >> 4;                 // 16-key steps
                     if (!(ok = mbar_wait(&bars[BAR_P_FULL + st], ph))) break;
                     if (!(ok = mbar_wait(&bars[BAR_V_FULL + st], ph))) break;
                     // the first O = P V of an item overwrites O: the previous item's must have been read out
                     if (cp.j == 0 && cp.item_no > 0 && !(ok = mbar_wait(&bars[BAR_O_FREE], (cp.item_no - 1) & 1))) break;
                     tc_fence_after();
-                    const uint32_t vb = v_lo + st * (kKVBytes >> 4);
+                    const uint32_t vb = (v_lo + st * (kKVBytes >> 4)) | (((32u << kv_box_sel(pv_valid)) * 8u) << 16);
                     const uint32_t pa = tb + st * kBN;
 #pragma unroll
                     for (int kk = 0; kk < kBN / 16; ++kk)                 // contraction over keys
@@ -597,9 +611,12 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
     SP_REQUIRE(((int64_t)n_heads * kHD * 2) % 16 == 0, SP_ERR_INVALID_ARG, "row stride must be a multiple of 16 bytes");
 
     TcParams p;
-    if (int rc = encode_rows_map(enc, &p.mq, q, lay->total_tokens, (int64_t)n_heads * kHD, kBM)) return rc;
-    if (int rc = encode_rows_map(enc, &p.mk, k, lay->total_tokens, (int64_t)n_kv_heads * kHD, kBN)) return rc;
-    if (int rc = encode_rows_map(enc, &p.mv, v, lay->total_tokens, (int64_t)n_kv_heads * kHD, kBN)) return rc;
+    for (int i = 0; i < 3; ++i)
+        if (int rc = encode_rows_map(enc, &p.mq[i], q, lay->total_tokens, (int64_t)n_heads * kHD, 32 << i)) return rc;
+    for (int i = 0; i < 2; ++i) {
+        if (int rc = encode_rows_map(enc, &p.mk[i], k, lay->total_tokens, (int64_t)n_kv_heads * kHD, 32 << i)) return rc;
+        if (int rc = encode_rows_map(enc, &p.mv[i], v, lay->total_tokens, (int64_t)n_kv_heads * kHD, 32 << i)) return rc;
+    }
 
     TcHeader *hdr = static_cast<TcHeader *>(ws);
     TcTile *tiles = reinterpret_cast<TcTile *>(static_cast<char *>(ws) + 256);
