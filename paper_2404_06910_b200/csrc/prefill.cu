@@ -1,4 +1,6 @@
 // sp_superpose_prefill entry point: argument checks and kernel selection.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace sp {
@@ -9,13 +11,17 @@ size_t prefill_tc_workspace_bytes(int n_prompts, int n_paths, int max_pre_len, i
 int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layout *lay, int n_heads,
                       int n_kv_heads, float scale, int rows, void *out, float *lse, void *ws,
                       size_t ws_bytes, cudaStream_t st);
+size_t prefill_qonly_workspace_bytes(int n_prompts, int n_paths, int max_pre_len, int max_path_len);
+int launch_prefill_qonly(const void *q, const void *k, const void *v, const sp_layout *lay, int n_heads,
+                         int n_kv_heads, float scale, void *out, float *lse, void *ws, cudaStream_t st);
 }  // namespace sp
 
 extern "C" size_t sp_prefill_workspace_bytes(int n_prompts, int n_paths, int max_pre_len,
                                              int max_path_len, int n_heads, int head_dim, int dtype)
 {
-    if (dtype == SP_BF16 && head_dim == 128)
-        return sp::prefill_tc_workspace_bytes(n_prompts, n_paths, max_pre_len, max_path_len, n_heads);
+    if (dtype == SP_BF16 && head_dim == 128)      // enough for either rows mode
+        return std::max(sp::prefill_tc_workspace_bytes(n_prompts, n_paths, max_pre_len, max_path_len, n_heads),
+                        sp::prefill_qonly_workspace_bytes(n_prompts, n_paths, max_pre_len, max_path_len));
     return 256;
 }
 
@@ -44,6 +50,8 @@ extern "C" int sp_superpose_prefill(const void *q, const void *k, const void *v,
                "sp_superpose_prefill: workspace of %zu bytes (256-byte aligned) required", need);
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dtype == SP_BF16 && head_dim == 128 && rows == SP_ROWS_QUERY_ONLY)
+        return launch_prefill_qonly(q, k, v, lay, n_heads, n_kv_heads, scale, out, lse, ws, st);
     if (dtype == SP_BF16 && head_dim == 128)
         return launch_prefill_tc(q, k, v, lay, n_heads, n_kv_heads, scale, rows, out, lse, ws, ws_bytes, st);
     SP_CUDA(cudaMemsetAsync(ws, 0, 256, st));

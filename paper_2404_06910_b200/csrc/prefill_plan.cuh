@@ -1,0 +1,91 @@
+// Tile list shared by the tensor-core prefill kernels: a one-block plan kernel turns the ragged
+// fork-join layout (Section 3.2) into query tiles of a given height, each knowing its segment,
+// its offset inside it and its prompt's fully visible preamble.
+#pragma once
+#include "common.cuh"
+
+namespace sp {
+
+struct TcTile {                       // one query tile (shared by all heads)
+    int32_t q_row;                    // packed row of the tile's first query row
+    int32_t n_rows;                   // valid rows in the tile (1..tile height)
+    int32_t q_off;                    // offset of the first row inside its segment
+    int32_t own_row;                  // packed row of the segment's first row
+    int32_t pre_row, pre_len;         // fully visible prefix (the prompt's preamble), may be empty
+    int32_t pad0, pad1;
+};
+
+struct TcHeader {                     // start of the workspace
+    uint32_t status;
+    uint32_t n_tiles;
+};
+
+// ---- plan: ragged layout -> tile list ---------------------------------------------------
+struct PlanArgs {
+    const int32_t *ppo, *pre_start, *pre_len, *path_start, *doc_len, *qry_len;
+    int n_prompts, n_paths, rows_mode;
+    int tile_rows;                    // query rows per tile
+    TcHeader *hdr;
+    TcTile *tiles;
+};
+
+static __global__ void __launch_bounds__(1024) prefill_plan_kernel(const PlanArgs a)
+{
+    __shared__ int warp_tot[32];
+    __shared__ int running;
+    if (threadIdx.x == 0) running = 0;
+    __syncthreads();
+    const int n_seq = a.n_prompts + a.n_paths;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int base = 0; base < n_seq; base += 1024) {
+        const int s = base + threadIdx.x;
+        int first = 0, rows = 0, own_row = 0, pre_row = 0, pre_n = 0;
+        if (s < a.n_prompts) {
+            if (a.rows_mode == SP_ROWS_ALL) { rows = a.pre_len[s]; own_row = a.pre_start[s]; }
+        } else if (s < n_seq) {
+            const int i = s - a.n_prompts;
+            int lo = 0, hi = a.n_prompts - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (a.ppo[mid] <= i) lo = mid; else hi = mid - 1;
+            }
+            pre_row = a.pre_start[lo]; pre_n = a.pre_len[lo];
+            own_row = a.path_start[i];
+            first = a.rows_mode == SP_ROWS_QUERY_ONLY ? a.doc_len[i] : 0;
+            rows = a.doc_len[i] + a.qry_len[i] - first;
+        }
+        const int nt = (rows + a.tile_rows - 1) / a.tile_rows;
+        int incl = nt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        int before = running;
+        for (int w = 0; w < warp; ++w) before += warp_tot[w];
+        int off = before + incl - nt;
+        for (int t = 0; t < nt; ++t) {
+            TcTile tl;
+            tl.q_off = first + t * a.tile_rows;
+            tl.q_row = own_row + tl.q_off;
+            tl.n_rows = min(a.tile_rows, rows - t * a.tile_rows);
+            tl.own_row = own_row;
+            tl.pre_row = pre_row; tl.pre_len = pre_n; tl.pad0 = 0; tl.pad1 = 0;
+            a.tiles[off + t] = tl;
+        }
+        __syncthreads();
+        if (threadIdx.x == 1023) running = before + incl;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) a.hdr->n_tiles = (uint32_t)running;
+}
+
+static inline int64_t plan_max_tiles(int n_prompts, int n_paths, int max_pre_len, int max_path_len, int tile_rows)
+{
+    return (int64_t)n_prompts * ((max_pre_len + tile_rows - 1) / tile_rows) +
+           (int64_t)n_paths * ((max_path_len + tile_rows - 1) / tile_rows);
+}
+
+}  // namespace sp

@@ -20,6 +20,7 @@
 #include <cstdlib>
 
 #include "common.cuh"
+#include "prefill_plan.cuh"
 #include "tc_ptx.cuh"
 
 namespace sp {
@@ -45,20 +46,6 @@ __device__ __forceinline__ float ex2(float x)
     return y;
 }
 
-struct TcTile {                       // one 128-row query tile (shared by all heads)
-    int32_t q_row;                    // packed row of the tile's first query row
-    int32_t n_rows;                   // valid rows in the tile (1..128)
-    int32_t q_off;                    // offset of the first row inside its segment
-    int32_t own_row;                  // packed row of the segment's first row
-    int32_t pre_row, pre_len;         // fully visible prefix (the prompt's preamble), may be empty
-    int32_t pad0, pad1;
-};
-
-struct TcHeader {                     // start of the workspace
-    uint32_t status;
-    uint32_t n_tiles;
-};
-
 // Tiles with few valid rows are fetched through tensor maps with shorter boxes (32 or 64 rows
 // instead of 128 / 64), so that ragged tails and query-only tiles do not pull in rows nobody
 // needs.  A box lands as two swizzled halves of box_rows x 128 bytes each.
@@ -77,67 +64,6 @@ struct TcParams {
     float scale_log2e;
     int stall_producer;               // test hook: the producer issues no load, so every wait runs out
 };
-
-// ---- plan: ragged layout -> tile list ---------------------------------------------------
-struct PlanArgs {
-    const int32_t *ppo, *pre_start, *pre_len, *path_start, *doc_len, *qry_len;
-    int n_prompts, n_paths, rows_mode;
-    TcHeader *hdr;
-    TcTile *tiles;
-};
-
-__global__ void __launch_bounds__(1024) prefill_plan_kernel(const PlanArgs a)
-{
-    __shared__ int warp_tot[32];
-    __shared__ int running;
-    if (threadIdx.x == 0) running = 0;
-    __syncthreads();
-    const int n_seq = a.n_prompts + a.n_paths;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int base = 0; base < n_seq; base += 1024) {
-        const int s = base + threadIdx.x;
-        int first = 0, rows = 0, own_row = 0, pre_row = 0, pre_n = 0;
-        if (s < a.n_prompts) {
-            if (a.rows_mode == SP_ROWS_ALL) { rows = a.pre_len[s]; own_row = a.pre_start[s]; }
-        } else if (s < n_seq) {
-            const int i = s - a.n_prompts;
-            int lo = 0, hi = a.n_prompts - 1;
-            while (lo < hi) {
-                const int mid = (lo + hi + 1) >> 1;
-                if (a.ppo[mid] <= i) lo = mid; else hi = mid - 1;
-            }
-            pre_row = a.pre_start[lo]; pre_n = a.pre_len[lo];
-            own_row = a.path_start[i];
-            first = a.rows_mode == SP_ROWS_QUERY_ONLY ? a.doc_len[i] : 0;
-            rows = a.doc_len[i] + a.qry_len[i] - first;
-        }
-        const int nt = (rows + kBM - 1) / kBM;
-        int incl = nt;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        if (lane == 31) warp_tot[warp] = incl;
-        __syncthreads();
-        int before = running;
-        for (int w = 0; w < warp; ++w) before += warp_tot[w];
-        int off = before + incl - nt;
-        for (int t = 0; t < nt; ++t) {
-            TcTile tl;
-            tl.q_off = first + t * kBM;
-            tl.q_row = own_row + tl.q_off;
-            tl.n_rows = min(kBM, rows - t * kBM);
-            tl.own_row = own_row;
-            tl.pre_row = pre_row; tl.pre_len = pre_n; tl.pad0 = 0; tl.pad1 = 0;
-            a.tiles[off + t] = tl;
-        }
-        __syncthreads();
-        if (threadIdx.x == 1023) running = before + incl;
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) a.hdr->n_tiles = (uint32_t)running;
-}
 
 // Key tile j of a query tile: preamble tiles first, then the segment's own rows up to the
 // tile's last valid query row.
@@ -586,7 +512,7 @@ static int encode_rows_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, 
 
 static int64_t max_tiles(int n_prompts, int n_paths, int max_pre_len, int max_path_len)
 {
-    return (int64_t)n_prompts * ((max_pre_len + kBM - 1) / kBM) + (int64_t)n_paths * ((max_path_len + kBM - 1) / kBM);
+    return plan_max_tiles(n_prompts, n_paths, max_pre_len, max_path_len, kBM);
 }
 
 size_t prefill_tc_workspace_bytes(int n_prompts, int n_paths, int max_pre_len, int max_path_len, int)
@@ -625,7 +551,7 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
     PlanArgs pa;
     pa.ppo = lay->prompt_path_off; pa.pre_start = lay->pre_start; pa.pre_len = lay->pre_len;
     pa.path_start = lay->path_start; pa.doc_len = lay->doc_len; pa.qry_len = lay->qry_len;
-    pa.n_prompts = lay->n_prompts; pa.n_paths = lay->n_paths; pa.rows_mode = rows;
+    pa.n_prompts = lay->n_prompts; pa.n_paths = lay->n_paths; pa.rows_mode = rows; pa.tile_rows = kBM;
     pa.hdr = hdr; pa.tiles = tiles;
     prefill_plan_kernel<<<1, 1024, 0, st>>>(pa);
     SP_CUDA(cudaGetLastError());
