@@ -23,7 +23,7 @@ constexpr int kQN = 32;               // keys per tile
 constexpr int kQD = 128;              // head_dim
 constexpr int kQStages = 3;
 constexpr int kQThreads = 64;         // two warps x 16 query rows
-constexpr int kQBlocksPerSM = 3;
+constexpr int kQBlocksPerSM = 4;
 constexpr int kRowB = kQD * 2;        // bytes of one (token, head) row
 constexpr int kTileB = kQN * kRowB;   // 8 KB: one K or V tile, also one Q tile
 constexpr float kLog2eQ = 1.4426950408889634f;
@@ -151,8 +151,7 @@ __global__ void __launch_bounds__(kQThreads, kQBlocksPerSM) prefill_qonly_kernel
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char *sK = smem;                               // [stages] 32 keys x 256 B
     unsigned char *sV = sK + kQStages * kTileB;             // [stages]
-    unsigned char *sQ = sV + kQStages * kTileB;             // [2] by item parity
-    unsigned char *sO = sQ + 2 * kTileB;                    // [2 warps] 16 rows x 256 B, output staging
+    unsigned char *sQ = sV + kQStages * kTileB;             // one item's 32 query rows
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tig = lane & 3;
@@ -163,40 +162,47 @@ __global__ void __launch_bounds__(kQThreads, kQBlocksPerSM) prefill_qonly_kernel
     lc.init(p.tiles, n_items, p.n_heads);
     cc = lc;
 
-    auto issue = [&]() {
-        if (lc.valid) {
-            const int st = lc.g % kQStages;
-            const QKv kt = lc.kv();
-            const int64_t col = (int64_t)(lc.h / p.kv_group) * kRowB;
-            if (lc.j == 0)
-                load_rows(sQ + (lc.item_no & 1) * kTileB, p.q + (int64_t)lc.h * kRowB, q_pitch, lc.t.q_row, lc.t.n_rows);
-            load_rows(sK + st * kTileB, p.k + col, kv_pitch, kt.row0, kt.n_valid);
-            load_rows(sV + st * kTileB, p.v + col, kv_pitch, kt.row0, kt.n_valid);
-            lc.next();
-        }
-        cp_async_commit();            // one group per slot, empty or not, so the wait count stays fixed
+    // Fetches run up to kQStages - 1 tiles ahead of the arithmetic, one cp.async group per tile.
+    // A new item's Q may replace the previous one only once both warps hold that one in
+    // registers (q_held: the last item whose Q fragments were loaded); until then the fetch
+    // cursor waits, which only happens behind items of one or two key tiles.
+    int q_held = -1;
+    auto fetch_one = [&]() {
+        const int st = lc.g % kQStages;
+        const QKv kt = lc.kv();
+        const int64_t col = (int64_t)(lc.h / p.kv_group) * kRowB;
+        if (lc.j == 0)
+            load_rows(sQ, p.q + (int64_t)lc.h * kRowB, q_pitch, lc.t.q_row, lc.t.n_rows);
+        load_rows(sK + st * kTileB, p.k + col, kv_pitch, kt.row0, kt.n_valid);
+        load_rows(sV + st * kTileB, p.v + col, kv_pitch, kt.row0, kt.n_valid);
+        cp_async_commit();
+        lc.next();
     };
-#pragma unroll
-    for (int s = 0; s < kQStages - 1; ++s) issue();
+    auto q_slot_busy = [&]() { return lc.j == 0 && (int)lc.item_no > q_held + 1; };
+    // prologue: one tile fewer than later on, no stage has been consumed yet
+    while (lc.valid && lc.g < kQStages - 1 && !q_slot_busy()) fetch_one();
 
     uint32_t qf[kQD / 16][4];        // this warp's 16 query rows as A fragments
     float o[kQD / 8][4];             // O accumulator: 16 rows x 128 columns
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // rows gid and gid + 8
 
     while (cc.valid) {
-        cp_async_wait<kQStages - 2>();
-        __syncthreads();             // tile cc.g has landed for every thread; the stage of tile cc.g - 1 is free
+        // tile cc.g must have landed: all groups but the ones of the tiles fetched after it
+        const int pend = (int)(lc.g - cc.g) - 1;
+        if (pend >= 2) cp_async_wait<2>(); else if (pend == 1) cp_async_wait<1>(); else cp_async_wait<0>();
+        __syncthreads();             // ... for every thread; and the stage of tile cc.g - 1 is free
         if (cc.j == 0) {
-            const uint32_t qb = smem_addr(sQ + (cc.item_no & 1) * kTileB);
+            const uint32_t qb = smem_addr(sQ);
 #pragma unroll
             for (int ks = 0; ks < kQD / 16; ++ks)
                 ldsm_x4(qb + sw_off(warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, ks * 2 + (lane >> 4)), qf[ks]);
 #pragma unroll
             for (int i = 0; i < kQD / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
             m_run[0] = m_run[1] = -INFINITY; l_run[0] = l_run[1] = 0.f;
-            __syncthreads();         // both warps hold their Q before the slot two items on is refilled
+            __syncthreads();         // both warps hold their Q before the next item's may be fetched
+            q_held = (int)cc.item_no;
         }
-        issue();
+        while (lc.valid && lc.g < cc.g + kQStages && !q_slot_busy()) fetch_one();
 
         const int st = cc.g % kQStages;
         const QKv kt = cc.kv();
@@ -266,7 +272,10 @@ __global__ void __launch_bounds__(kQThreads, kQBlocksPerSM) prefill_qonly_kernel
 
         if (cc.last_of_item()) {
             // ---- O / l -> bf16 -> staging -> 16-byte stores; log-sum-exp
-            unsigned char *stage = sO + warp * (16 * kRowB);
+            // staging reuses this tile's K stage: every S = Q K^T of the block that reads it is
+            // behind the barrier below, and the stage is refilled only after the next block barrier
+            __syncthreads();
+            unsigned char *stage = sK + st * kTileB + warp * (16 * kRowB);
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
                 float l = l_run[hh];
@@ -328,7 +337,7 @@ int launch_prefill_qonly(const void *q, const void *k, const void *v, const sp_l
     p.hdr = hdr; p.tiles = tiles;
     p.n_heads = n_heads; p.n_kv_heads = n_kv_heads; p.kv_group = n_heads / n_kv_heads;
     p.total_tokens = lay->total_tokens; p.scale_log2e = scale * kLog2eQ;
-    const int smem = (2 * kQStages + 2) * kTileB + 2 * 16 * kRowB;
+    const int smem = (2 * kQStages + 1) * kTileB;
     SP_CUDA(cudaFuncSetAttribute(prefill_qonly_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int grid = (int)std::min<int64_t>(items, (int64_t)kQBlocksPerSM * kNumSMs);
     prefill_qonly_kernel<<<grid, kQThreads, smem, st>>>(p);
