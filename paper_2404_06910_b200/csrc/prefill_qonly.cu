@@ -16,8 +16,6 @@
 
 namespace sp {
 
-namespace {
-
 constexpr int kQM = 32;               // query rows per item
 constexpr int kQN = 32;               // keys per tile
 constexpr int kQD = 128;              // head_dim
@@ -305,8 +303,6 @@ __global__ void __launch_bounds__(kQThreads, kQBlocksPerSM) prefill_qonly_kernel
     }
     cp_async_wait<0>();
 }
-
-}  // namespace
 
 size_t prefill_qonly_workspace_bytes(int n_prompts, int n_paths, int max_pre_len, int max_path_len)
 {

@@ -50,7 +50,32 @@ def test_full_size_sampled(cfg):
         den = np.linalg.norm(ref_o.reshape(len(rows), -1), axis=1) + 1e-6
         assert (num / den).max() <= 5e-2
         np.testing.assert_allclose(got_l, ref_l, atol=2e-2)
-    del out, lse, qd
+    # ---- the same prompts in cached / online mode: only query rows are produced -----------
+    out_q = torch.full_like(qd, float("nan"))
+    lse_q = torch.full((H, lay.total_tokens), float("nan"), device="cuda")
+    sp.sp_superpose_prefill(qd, kd, vd, dl, scale, out_q, lse_q, ws, rows=sp.SP_ROWS_QUERY_ONLY)
+    sp.sp_check_status(ws)
+    is_q = np.zeros(lay.total_tokens, bool)
+    for i in range(lay.n_paths):
+        s0 = lay.path_start[i] + lay.doc_len[i]
+        is_q[s0:s0 + lay.qry_len[i]] = True
+    is_qd = torch.from_numpy(is_q).cuda()
+    assert not bool(torch.isnan(out_q[is_qd]).any()), "query rows left unwritten"
+    assert bool(torch.isnan(out_q[~is_qd]).all()), "non-query rows must stay untouched"
+    # both modes compute the same rows from the same inputs: they must agree to bf16 rounding
+    diff = (out_q[is_qd].float() - out[is_qd].float()).abs().max().item()
+    assert diff <= 2e-2 * out[is_qd].float().abs().max().item()
+    for b in prompts[:2]:
+        p0, p1 = int(lay.prompt_path_off[b]), int(lay.prompt_path_off[b + 1])
+        paths = sorted(set([p0, p1 - 1, int(rng.integers(p0, p1))]))
+        sub, rows, _ = sub_problem(lay, b, paths)
+        ref_o, ref_l = oracle.prefill(f32(q[rows]), f32(k[rows]), f32(v[rows]), sub, scale)
+        sel = is_q[rows]
+        got_o = f32(out_q[torch.from_numpy(rows).cuda()])
+        got_l = lse_q[:, torch.from_numpy(rows).cuda()].cpu().numpy()
+        assert rel_l2(got_o[sel], ref_o[sel]) <= 1e-2
+        np.testing.assert_allclose(got_l[:, sel], ref_l[:, sel], atol=2e-2)
+    del out, lse, qd, out_q, lse_q
 
     # ---- decode: all prompts on the GPU, sampled prompts in the oracle -----------------
     scores = rng.standard_normal(lay.n_paths).astype(np.float32)

@@ -178,6 +178,58 @@ def test_prefill_query_only_rows(dtype, D):
     np.testing.assert_allclose(got_l[:, is_q], ref_l[:, is_q], atol=1e-5 if dtype == "f32" else 2e-2)
 
 
+def _query_row_mask(lay):
+    is_q = np.zeros(lay.total_tokens, bool)
+    for i in range(lay.n_paths):
+        s = lay.path_start[i] + lay.doc_len[i]
+        is_q[s:s + lay.qry_len[i]] = True
+    return is_q
+
+
+@pytest.mark.parametrize("case", ["ragged", "long_queries", "no_preamble_short", "many_paths"])
+def test_prefill_query_only_ragged(case):
+    """Query rows only (bf16, head_dim 128): query lengths around and beyond the 32-row item,
+    empty documents and preambles, items of one or two key tiles behind longer ones, grouped
+    heads; per-row check, untouched non-query rows, and bit-identical repeats."""
+    rng = np.random.default_rng(11)
+    if case == "ragged":
+        lay = build_layout([0, 5, 40, 130], [[1, 15, 16, 31], [17, 127, 0], [128, 129], [300, 2, 64]],
+                           [[1, 1, 2, 32], [3, 33, 8], [7, 24], [31, 1, 64]])
+        H, Hkv = 4, 2
+    elif case == "long_queries":
+        lay = build_layout([33], [[200, 10, 0]], [[100, 65, 140]])
+        H, Hkv = 2, 2
+    elif case == "no_preamble_short":
+        # items with one key tile (<= 32 keys in all) mixed with long ones, 2 heads
+        docs = [int(x) for x in rng.integers(0, 20, 300)]
+        docs[::7] = [250] * len(docs[::7])
+        lay = build_layout([0], [docs], [[int(x) for x in rng.integers(1, 12, 300)]])
+        H, Hkv = 2, 1
+    else:
+        lay = build_layout([32] * 3, [[int(x) for x in rng.integers(64, 257, 40)] for _ in range(3)], [[24] * 40] * 3)
+        H, Hkv = 8, 8
+    T, D = lay.total_tokens, 128
+    q, k, v = _randn((T, H, D), "bf16", 21), _randn((T, Hkv, D), "bf16", 22), _randn((T, Hkv, D), "bf16", 23)
+    gain = np.ones(T, np.float32)
+    gain[T // 3: 2 * T // 3] = 4.0
+    q = (q.float() * torch.from_numpy(gain)[:, None, None]).to(q.dtype)
+    scale = 1 / math.sqrt(D)
+    ref_o, ref_l = oracle.prefill(f32(q), f32(k), f32(v), lay, scale)
+    got_o, got_l = _prefill_gpu(q, k, v, lay, scale, rows=sp.SP_ROWS_QUERY_ONLY)
+    is_q = _query_row_mask(lay)
+    assert np.isnan(got_o[~is_q]).all(), "non-query rows must stay untouched"
+    assert not np.isnan(got_o[is_q]).any(), "query rows left unwritten"
+    num = np.linalg.norm((got_o - ref_o)[is_q].reshape(int(is_q.sum()), -1), axis=1)
+    den = np.linalg.norm(ref_o[is_q].reshape(int(is_q.sum()), -1), axis=1) + 1e-6
+    assert rel_l2(got_o[is_q], ref_o[is_q]) <= TOL["bf16"]
+    assert (num / den).max() <= 5 * TOL["bf16"]
+    np.testing.assert_allclose(got_l[:, is_q], ref_l[:, is_q], atol=2e-2)
+    for _ in range(3):
+        again_o, again_l = _prefill_gpu(q, k, v, lay, scale, rows=sp.SP_ROWS_QUERY_ONLY)
+        np.testing.assert_array_equal(again_o[is_q], got_o[is_q])
+        np.testing.assert_array_equal(again_l[:, is_q], got_l[:, is_q])
+
+
 def test_prefill_is_deterministic():
     cfg = CONFIGS[1]
     lay = draw_lengths(cfg)
