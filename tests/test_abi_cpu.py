@@ -109,3 +109,14 @@ def test_workspace_sizes_are_sane():
     assert lib.sp_decode_workspace_bytes(1, 32, 128) % 256 == 0
     assert lib.sp_decode_workspace_bytes(64, 32, 128) >= 256
     assert lib.sp_prefill_workspace_bytes(1, 20, 32, 184, 32, 128, sp.SP_BF16) >= 256
+
+
+def test_next_round_layout_moves_kept_documents_into_the_prefix():
+    import numpy as np
+    from workloads import build_layout, next_round_layout
+    lay = build_layout([3, 0], [[10, 20, 30], [5, 6]], [[4, 4, 4], [2, 2]])
+    nxt = next_round_layout(lay, np.array([[2, 0], [4, -1]]))
+    assert list(nxt.pre_len) == [3 + 30 + 10, 6]
+    assert list(nxt.doc_len) == [20, 5] and list(nxt.qry_len) == [4, 2]
+    assert list(nxt.prompt_path_off) == [0, 1, 2]
+    assert nxt.total_tokens == 43 + 24 + 6 + 7

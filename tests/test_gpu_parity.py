@@ -13,7 +13,7 @@ import oracle
 import paper_2404_06910_b200 as sp
 from helpers import dev, f32, positions_for, rel_l2, workspace
 from workloads import (CONFIGS, build_layout, draw_decode_inputs, draw_lengths, draw_logits,
-                       draw_prior_weight, draw_qkv, draw_targets)
+                       draw_prior_weight, draw_qkv, draw_targets, next_round_layout)
 
 pytestmark = pytest.mark.gpu
 
@@ -502,3 +502,67 @@ def test_chain_rope_prefill_scores_topk_decode(cfg):
         tk_ref[:, t] = rnd(oracle.rope(np.ascontiguousarray(tk_ref[:, t]), tpos, base=cfg.rope_base))
         ref_d, _ = oracle.pruned_decode(qt_ref, k_r, f32(v), lay, kept_h, tk_ref, tv_ref, tl, scale)
         assert rel_l2(f32(o), ref_d) <= TOL[cfg.dtype] * (1 if cfg.dtype == "bf16" else 3)
+
+
+def test_iterative_superposition_rounds():
+    """Section 4.3's iterative variant, t = 3 rounds with k = 2: each round is a fork-join prefill
+    over the remaining documents behind a shared prefix that has grown by the documents kept so
+    far, scored and pruned; the response then attends to the final prefix plus the last kept paths.
+    Every round's device results are checked against the oracle on the same layout."""
+    cfg = CONFIGS[1]
+    H, Hkv, D, k_top = 8, 4, 128, 2
+    rng = np.random.default_rng(99)
+    lay = build_layout([20, 7], [list(rng.integers(40, 200, 9)), list(rng.integers(40, 200, 7))], [[12] * 9, [12] * 7])
+    scale = 1 / math.sqrt(D)
+    for rnd_no in range(3):
+        B, T = lay.n_prompts, lay.total_tokens
+        q, k, v = _randn((T, H, D), "bf16", 50 + rnd_no), _randn((T, Hkv, D), "bf16", 60 + rnd_no), _randn((T, Hkv, D), "bf16", 70 + rnd_no)
+        pos, _ = positions_for(lay, lambda P, L, Q: sp.sp_positions(P, L, Q))
+        pos_ref, _ = positions_for(lay, lambda P, L, Q: oracle.positions(P, L, Q))
+        np.testing.assert_array_equal(pos, pos_ref)
+        dl = sp.DeviceLayout.from_host(lay)
+        qd, kd, vd = dev(q), dev(k), dev(v)
+        sp.sp_rope_apply(qd, dev(pos), H, D)
+        sp.sp_rope_apply(kd, dev(pos), Hkv, D)
+        out = torch.full_like(qd, float("nan"))
+        ws = workspace(sp.sp_prefill_workspace_bytes(dl, H, D, sp.SP_BF16))
+        sp.sp_superpose_prefill(qd, kd, vd, dl, scale, out, None, ws)
+        sp.sp_check_status(ws)
+        bf = lambda a: torch.from_numpy(a).bfloat16().float().numpy()
+        q_r, k_r = bf(oracle.rope(f32(q), pos_ref)), bf(oracle.rope(f32(k), pos_ref))
+        ref_o, _ = oracle.prefill(q_r, k_r, f32(v), lay, scale)
+        assert rel_l2(f32(out), ref_o) <= TOL["bf16"]
+        # the same round in cached mode (query rows only) agrees on the query rows
+        out_q = torch.full_like(qd, float("nan"))
+        sp.sp_superpose_prefill(qd, kd, vd, dl, scale, out_q, None, ws, rows=sp.SP_ROWS_QUERY_ONLY)
+        is_q = _query_row_mask(lay)
+        assert rel_l2(f32(out_q)[is_q], ref_o[is_q]) <= TOL["bf16"]
+
+        R = int(lay.qry_len.sum())
+        logits = _randn((R, 777), "bf16", 80 + rnd_no, 3.0)
+        tgt = rng.integers(0, 777, R).astype(np.int32)
+        off = lay.query_row_offsets()
+        weight = (1.0 / np.maximum(lay.qry_len, 1)).astype(np.float32)
+        prior = rng.normal(-2.5, 0.25, lay.n_paths).astype(np.float32)
+        scores = torch.empty(lay.n_paths, device="cuda")
+        sp.sp_path_scores(dev(logits), dev(tgt), dev(off), scores, dev(prior), dev(weight), None,
+                          workspace(sp.sp_path_scores_workspace_bytes(R)))
+        ref_s, _ = oracle.path_scores(f32(logits), tgt, off, prior, weight)
+        np.testing.assert_allclose(scores.cpu().numpy(), ref_s, atol=1e-3)
+        kept = torch.empty((B, k_top), dtype=torch.int32, device="cuda")
+        sp.sp_prune_topk(scores, dl.prompt_path_off, k_top, kept)
+        ref_kept, _ = oracle.prune_topk(scores.cpu().numpy(), lay.prompt_path_off, k_top)
+        np.testing.assert_array_equal(kept.cpu().numpy(), ref_kept)     # same scores in: bit-exact
+        if rnd_no < 2:
+            nxt = next_round_layout(lay, ref_kept)
+            assert nxt.n_paths == lay.n_paths - B * k_top
+            assert nxt.total_tokens == lay.total_tokens - sum(int(lay.qry_len[i]) for i in ref_kept.ravel())
+            lay = nxt
+    # response step on the last round's tensors: prefix (preamble + 4 documents kept earlier) + 2 kept paths
+    dq, tk, tv = _randn((B, H, D), "bf16", 90), _randn((B, 1, Hkv, D), "bf16", 91), _randn((B, 1, Hkv, D), "bf16", 92)
+    o = torch.empty((B, H, D), dtype=torch.bfloat16, device="cuda")
+    tl = np.ones(B, np.int32)
+    sp.sp_pruned_decode(dev(dq), kd, vd, dl, kept, k_top, dev(tk), dev(tv), dev(tl), 1, scale, o, None,
+                        workspace(sp.sp_decode_workspace_bytes(B, H, D)))
+    ref_d, _ = oracle.pruned_decode(f32(dq), k_r, f32(v), lay, ref_kept, f32(tk), f32(tv), tl, scale)
+    assert rel_l2(f32(o), ref_d) <= TOL["bf16"]

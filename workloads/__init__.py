@@ -6,7 +6,7 @@ CPU oracle and the CUDA library each implement those on their own and both are
 fed from here.
 """
 from .configs import CONFIGS, Config, get_config  # noqa: F401
-from .layout import Layout, build_layout, draw_lengths  # noqa: F401
+from .layout import Layout, build_layout, draw_lengths, next_round_layout  # noqa: F401
 from .tensors import (  # noqa: F401
     bf16_round,
     draw_decode_inputs,

@@ -90,3 +90,19 @@ def draw_lengths(cfg: Config, seed: int | None = None, n_prompts: int | None = N
     docs = [rng.integers(cfg.doc_len_min, cfg.doc_len_max + 1, size=cfg.n_docs) for _ in range(B)]
     qrys = [np.full(cfg.n_docs, cfg.qry_len) for _ in range(B)]
     return build_layout([cfg.pre_len] * B, docs, qrys)
+
+
+def next_round_layout(lay: Layout, kept: np.ndarray) -> Layout:
+    """Iterative superposition (Section 4.3): the documents kept in this round (global path
+    ids per prompt, -1 = none) join the prompt's shared prefix, in the order given; every other
+    path stays a path of the next round, with its own copy of the query."""
+    kept = np.asarray(kept).reshape(lay.n_prompts, -1)
+    pre, docs, qrys = [], [], []
+    for b in range(lay.n_prompts):
+        p0, p1 = int(lay.prompt_path_off[b]), int(lay.prompt_path_off[b + 1])
+        chosen = [int(i) for i in kept[b] if p0 <= int(i) < p1]
+        pre.append(int(lay.pre_len[b]) + sum(int(lay.doc_len[i]) for i in chosen))
+        rest = [i for i in range(p0, p1) if i not in chosen]
+        docs.append([int(lay.doc_len[i]) for i in rest])
+        qrys.append([int(lay.qry_len[i]) for i in rest])
+    return build_layout(pre, docs, qrys)
