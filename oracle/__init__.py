@@ -90,9 +90,10 @@ def _lay_args(lay):
     return arrs, [ctypes.c_int(lay.n_prompts)] + [_p(a) for a in arrs]
 
 
-def prefill(q, k, v, lay, scale, rows=None, want_lse=True):
+def prefill(q, k, v, lay, scale, rows=None, want_lse=True, pos=None, slopes=None):
     """q [T,H,D], k/v [T,Hkv,D] float32.  Returns (out [T,H,D], lse [H,T]).
-    With ``rows`` (int64 list) only those packed rows are computed; the rest stay 0."""
+    With ``rows`` (int64 list) only those packed rows are computed; the rest stay 0.
+    With ``pos`` [T] and ``slopes`` [H] the scores get the ALiBi bias -slope * |pos_q - pos_k|."""
     q, k, v = _f32(q), _f32(k), _f32(v)
     T, H, D = q.shape
     Hkv = k.shape[1]
@@ -101,9 +102,12 @@ def prefill(q, k, v, lay, scale, rows=None, want_lse=True):
     lse = np.zeros((H, T), dtype=np.float32) if want_lse else None
     keep, largs = _lay_args(lay)
     r = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
-    rc = _load().spo_prefill(_p(q), _p(k), _p(v), *largs, ctypes.c_int64(T), ctypes.c_int(H),
-                             ctypes.c_int(Hkv), ctypes.c_int(D), ctypes.c_double(scale),
-                             _p(r), ctypes.c_int64(0 if r is None else len(r)), _p(out), _p(lse))
+    ps = None if pos is None else _f32(pos)
+    sl = None if slopes is None else _f32(slopes)
+    assert (ps is None) == (sl is None) and (ps is None or (ps.shape == (T,) and sl.shape == (H,)))
+    rc = _load().spo_prefill_alibi(_p(q), _p(k), _p(v), *largs, ctypes.c_int64(T), ctypes.c_int(H),
+                                   ctypes.c_int(Hkv), ctypes.c_int(D), ctypes.c_double(scale), _p(ps), _p(sl),
+                                   _p(r), ctypes.c_int64(0 if r is None else len(r)), _p(out), _p(lse))
     _check(rc, "prefill")
     return out, lse
 
@@ -134,8 +138,10 @@ def prune_topk(scores, prompt_path_off, k):
     return idx, post
 
 
-def pruned_decode(q, k_cache, v_cache, lay, kept_idx, tail_k, tail_v, tail_len, scale):
-    """q [B,H,D]; caches [T,Hkv,D]; tail_k/v [B,cap,Hkv,D]; kept_idx [B,k]; tail_len [B]."""
+def pruned_decode(q, k_cache, v_cache, lay, kept_idx, tail_k, tail_v, tail_len, scale,
+                  q_pos=None, cache_pos=None, tail_pos=None, slopes=None):
+    """q [B,H,D]; caches [T,Hkv,D]; tail_k/v [B,cap,Hkv,D]; kept_idx [B,k]; tail_len [B].
+    ALiBi: q_pos [B], cache_pos [T], tail_pos [B,cap], slopes [H] (all or none)."""
     q, k_cache, v_cache = _f32(q), _f32(k_cache), _f32(v_cache)
     B, H, D = q.shape
     Hkv = k_cache.shape[1]
@@ -150,9 +156,14 @@ def pruned_decode(q, k_cache, v_cache, lay, kept_idx, tail_k, tail_v, tail_len, 
     out = np.zeros((B, H, D), dtype=np.float32)
     lse = np.zeros((B, H), dtype=np.float32)
     keep, largs = _lay_args(lay)
-    rc = _load().spo_pruned_decode(_p(q), _p(k_cache), _p(v_cache), *largs, _p(kept_idx), ctypes.c_int(k),
-                                   _p(tail_k), _p(tail_v), _p(tail_len), ctypes.c_int(cap),
-                                   ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D),
-                                   ctypes.c_double(scale), _p(out), _p(lse))
+    qp = None if slopes is None else _f32(q_pos)
+    cp = None if slopes is None else _f32(cache_pos)
+    tp = None if slopes is None else (_f32(tail_pos) if tail_pos is not None else np.zeros((B, cap), dtype=np.float32))
+    sl = None if slopes is None else _f32(slopes)
+    assert sl is None or (qp.shape == (B,) and cp.shape == (k_cache.shape[0],) and tp.shape == (B, cap) and sl.shape == (H,))
+    rc = _load().spo_pruned_decode_alibi(_p(q), _p(k_cache), _p(v_cache), *largs, _p(kept_idx), ctypes.c_int(k),
+                                         _p(tail_k), _p(tail_v), _p(tail_len), ctypes.c_int(cap),
+                                         ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D),
+                                         ctypes.c_double(scale), _p(qp), _p(cp), _p(tp), _p(sl), _p(out), _p(lse))
     _check(rc, "pruned_decode")
     return out, lse

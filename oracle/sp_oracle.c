@@ -166,10 +166,10 @@ static int fill_row_info(int n_prompts, const int32_t *ppo, const int32_t *pre_s
 }
 
 /* Dense softmax attention of one query vector over an explicit key list.
- * s_j = scale * <q, k_j>;  m = max_j s_j;  LSE = m + ln sum_j exp(s_j - m);
- * o = sum_j exp(s_j - LSE) v_j.  Two passes, double arithmetic.                     */
+ * s_j = scale * <q, k_j> (+ bias_j);  m = max_j s_j;  LSE = m + ln sum_j exp(s_j - m);
+ * o = sum_j exp(s_j - LSE) v_j.  Two passes, double arithmetic.  bias may be NULL.     */
 static void attend_one(const float *qv, const float *const *kptr, const float *const *vptr,
-                       int64_t nk, int D, double scale, double *s, float *o, float *lse)
+                       int64_t nk, int D, double scale, const double *bias, double *s, float *o, float *lse)
 {
     double m = -INFINITY;
     for (int64_t j = 0; j < nk; ++j) {
@@ -177,6 +177,7 @@ static void attend_one(const float *qv, const float *const *kptr, const float *c
         const float *kv = kptr[j];
         for (int d = 0; d < D; ++d) acc += (double)qv[d] * (double)kv[d];
         s[j] = acc * scale;
+        if (bias) s[j] += bias[j];
         if (s[j] > m) m = s[j];
     }
     double denom = 0.0;
@@ -208,14 +209,20 @@ static void attend_one(const float *qv, const float *const *kptr, const float *c
  * out: [T, H, D]; lse: [H, T] natural log, may be NULL.
  * rows/n_rows: optional list of packed rows to compute (others untouched); NULL = all.
  * Reading: scale is passed explicitly (the paper does not restate 1/sqrt(D)).
+ * ALiBi (Section 3.2.2 notes that real-valued positions are trivial for it): with pos [T] and
+ * slopes [H] given, score(r, c) gets the additive bias -slopes[h] * |pos[r] - pos[c]|, the
+ * linear distance penalty of ALiBi evaluated at the tokens' assigned (possibly fractional)
+ * positions.  pos == NULL: no bias.
  * ---------------------------------------------------------------------------------- */
-int spo_prefill(const float *q, const float *k, const float *v,
-                int n_prompts, const int32_t *ppo, const int32_t *pre_start,
-                const int32_t *pre_len, const int32_t *path_start, const int32_t *doc_len,
-                const int32_t *qry_len, int64_t T, int H, int Hkv, int D, double scale,
-                const int64_t *rows, int64_t n_rows, float *out, float *lse)
+int spo_prefill_alibi(const float *q, const float *k, const float *v,
+                      int n_prompts, const int32_t *ppo, const int32_t *pre_start,
+                      const int32_t *pre_len, const int32_t *path_start, const int32_t *doc_len,
+                      const int32_t *qry_len, int64_t T, int H, int Hkv, int D, double scale,
+                      const float *pos, const float *slopes,
+                      const int64_t *rows, int64_t n_rows, float *out, float *lse)
 {
     if (!q || !k || !v || !out || H <= 0 || Hkv <= 0 || H % Hkv || D <= 0 || D > 512) return -1;
+    if (pos && !slopes) return -1;
     row_info *info = (row_info *)malloc(sizeof(row_info) * (size_t)(T > 0 ? T : 1));
     if (!info) return -3;
     int rc = fill_row_info(n_prompts, ppo, pre_start, pre_len, path_start, doc_len, qry_len, T, info);
@@ -227,7 +234,7 @@ int spo_prefill(const float *q, const float *k, const float *v,
     {
         int64_t cap = 0;
         const float **kp = NULL, **vp = NULL;
-        double *s = NULL;
+        double *s = NULL, *bias = NULL;
 #pragma omp for schedule(dynamic, 4)
         for (int64_t ii = 0; ii < n; ++ii) {
             const int64_t r = rows ? rows[ii] : ii;
@@ -241,6 +248,7 @@ int spo_prefill(const float *q, const float *k, const float *v,
                 kp = (const float **)realloc((void *)kp, sizeof(float *) * (size_t)cap);
                 vp = (const float **)realloc((void *)vp, sizeof(float *) * (size_t)cap);
                 s = (double *)realloc(s, sizeof(double) * (size_t)cap);
+                bias = (double *)realloc(bias, sizeof(double) * (size_t)cap);
             }
             for (int h = 0; h < H; ++h) {
                 const int hk = h / group;
@@ -260,14 +268,30 @@ int spo_prefill(const float *q, const float *k, const float *v,
                         kp[c] = k + (kr * Hkv + hk) * D; vp[c] = v + (kr * Hkv + hk) * D;
                     }
                 }
-                attend_one(q + (r * H + h) * D, kp, vp, c, D, scale, s,
+                if (pos) {
+                    for (int64_t cc = 0; cc < c; ++cc) {
+                        const int64_t kr = ((kp[cc] - k) / D - hk) / Hkv;      /* packed row of key cc */
+                        bias[cc] = -(double)slopes[h] * fabs((double)pos[r] - (double)pos[kr]);
+                    }
+                }
+                attend_one(q + (r * H + h) * D, kp, vp, c, D, scale, pos ? bias : NULL, s,
                            out + (r * H + h) * D, lse ? lse + (int64_t)h * T + r : NULL);
             }
         }
-        free((void *)kp); free((void *)vp); free(s);
+        free((void *)kp); free((void *)vp); free(s); free(bias);
     }
     free(info);
     return err ? -2 : 0;
+}
+
+int spo_prefill(const float *q, const float *k, const float *v,
+                int n_prompts, const int32_t *ppo, const int32_t *pre_start,
+                const int32_t *pre_len, const int32_t *path_start, const int32_t *doc_len,
+                const int32_t *qry_len, int64_t T, int H, int Hkv, int D, double scale,
+                const int64_t *rows, int64_t n_rows, float *out, float *lse)
+{
+    return spo_prefill_alibi(q, k, v, n_prompts, ppo, pre_start, pre_len, path_start, doc_len, qry_len, T, H, Hkv,
+                             D, scale, NULL, NULL, rows, n_rows, out, lse);
 }
 
 /* ------------------------------------------------------------------------------------
@@ -377,16 +401,21 @@ int spo_prune_topk(const float *scores, const int32_t *ppo, int n_prompts, int k
  * before the call (Reading: the new token attends to itself, as in any causal LM).
  * q: [B, H, D]; k_cache, v_cache: [T, Hkv, D]; tail_k, tail_v: [B, tail_cap, Hkv, D];
  * kept_idx: [B, k] with -1 padding; out: [B, H, D]; lse: [B, H] or NULL.
+ * ALiBi: with slopes [H] given, key c gets the bias -slopes[h] * |q_pos[b] - pos(c)|, where
+ * pos(c) is cache_pos[row] for cache rows and tail_pos[b, j] for tail rows.  slopes == NULL:
+ * no bias.
  * ---------------------------------------------------------------------------------- */
-int spo_pruned_decode(const float *q, const float *k_cache, const float *v_cache,
-                      int n_prompts, const int32_t *ppo, const int32_t *pre_start,
-                      const int32_t *pre_len, const int32_t *path_start,
-                      const int32_t *doc_len, const int32_t *qry_len,
-                      const int32_t *kept_idx, int k, const float *tail_k, const float *tail_v,
-                      const int32_t *tail_len, int tail_cap, int H, int Hkv, int D,
-                      double scale, float *out, float *lse)
+int spo_pruned_decode_alibi(const float *q, const float *k_cache, const float *v_cache,
+                            int n_prompts, const int32_t *ppo, const int32_t *pre_start,
+                            const int32_t *pre_len, const int32_t *path_start,
+                            const int32_t *doc_len, const int32_t *qry_len,
+                            const int32_t *kept_idx, int k, const float *tail_k, const float *tail_v,
+                            const int32_t *tail_len, int tail_cap, int H, int Hkv, int D,
+                            double scale, const float *q_pos, const float *cache_pos,
+                            const float *tail_pos, const float *slopes, float *out, float *lse)
 {
     if (!q || !k_cache || !v_cache || !out || H <= 0 || Hkv <= 0 || H % Hkv || D <= 0 || D > 512) return -1;
+    if (slopes && (!q_pos || !cache_pos)) return -1;
     if (k < 0 || (k > 0 && !kept_idx)) return -1;
     const int group = H / Hkv;
     int err = 0;
@@ -412,7 +441,8 @@ int spo_pruned_decode(const float *q, const float *k_cache, const float *v_cache
             const float **kp = (const float **)malloc(sizeof(float *) * (size_t)nk);
             const float **vp = (const float **)malloc(sizeof(float *) * (size_t)nk);
             double *s = (double *)malloc(sizeof(double) * (size_t)nk);
-            int64_t c = 0;
+            double *bias = (double *)malloc(sizeof(double) * (size_t)nk);
+            int64_t c = 0, n_cache;
             for (int j = 0; j < pre_len[b]; ++j, ++c) {
                 const int64_t kr = (int64_t)pre_start[b] + j;
                 kp[c] = k_cache + (kr * Hkv + hk) * D; vp[c] = v_cache + (kr * Hkv + hk) * D;
@@ -425,14 +455,36 @@ int spo_pruned_decode(const float *q, const float *k_cache, const float *v_cache
                     kp[c] = k_cache + (kr * Hkv + hk) * D; vp[c] = v_cache + (kr * Hkv + hk) * D;
                 }
             }
+            n_cache = c;
             for (int j = 0; j < tl; ++j, ++c) {
                 const int64_t kr = (int64_t)b * tail_cap + j;
                 kp[c] = tail_k + (kr * Hkv + hk) * D; vp[c] = tail_v + (kr * Hkv + hk) * D;
             }
-            attend_one(q + ((int64_t)b * H + h) * D, kp, vp, c, D, scale, s,
+            if (slopes) {
+                for (int64_t cc = 0; cc < c; ++cc) {
+                    const float *base = cc < n_cache ? k_cache : tail_k;
+                    const int64_t kr = ((kp[cc] - base) / D - hk) / Hkv;
+                    const double pk = cc < n_cache ? (double)cache_pos[kr] : (double)tail_pos[kr];
+                    bias[cc] = -(double)slopes[h] * fabs((double)q_pos[b] - pk);
+                }
+            }
+            attend_one(q + ((int64_t)b * H + h) * D, kp, vp, c, D, scale, slopes ? bias : NULL, s,
                        out + ((int64_t)b * H + h) * D, lse ? lse + b * H + h : NULL);
-            free((void *)kp); free((void *)vp); free(s);
+            free((void *)kp); free((void *)vp); free(s); free(bias);
         }
     }
     return err ? -2 : 0;
+}
+
+int spo_pruned_decode(const float *q, const float *k_cache, const float *v_cache,
+                      int n_prompts, const int32_t *ppo, const int32_t *pre_start,
+                      const int32_t *pre_len, const int32_t *path_start,
+                      const int32_t *doc_len, const int32_t *qry_len,
+                      const int32_t *kept_idx, int k, const float *tail_k, const float *tail_v,
+                      const int32_t *tail_len, int tail_cap, int H, int Hkv, int D,
+                      double scale, float *out, float *lse)
+{
+    return spo_pruned_decode_alibi(q, k_cache, v_cache, n_prompts, ppo, pre_start, pre_len, path_start, doc_len,
+                                   qry_len, kept_idx, k, tail_k, tail_v, tail_len, tail_cap, H, Hkv, D, scale,
+                                   NULL, NULL, NULL, NULL, out, lse);
 }

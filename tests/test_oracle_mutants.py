@@ -35,6 +35,14 @@ MUTANTS = [
     ("score_counts_ignored_rows", "if (y == -1) { if (row_logp) row_logp[t] = 0.0f; continue; }", "if (y == -1) { if (row_logp) row_logp[t] = 0.0f; sum += -1.0; continue; }", "path_scores"),
     ("topk_keeps_smallest", "if (s[a] != s[b]) return s[a] > s[b];", "if (s[a] != s[b]) return s[a] < s[b];", "topk"),
     ("topk_ties_to_higher_index", "if (s[a] != s[b]) return s[a] > s[b];\n    return a < b;", "if (s[a] != s[b]) return s[a] > s[b];\n    return a > b;", "topk"),
+    ("alibi_sign_flipped", "bias[cc] = -(double)slopes[h] * fabs((double)pos[r] - (double)pos[kr]);",
+     "bias[cc] = (double)slopes[h] * fabs((double)pos[r] - (double)pos[kr]);", "alibi"),
+    ("alibi_position_of_wrong_key", "bias[cc] = -(double)slopes[h] * fabs((double)pos[r] - (double)pos[kr]);",
+     "bias[cc] = -(double)slopes[h] * fabs((double)pos[r] - (double)pos[cc]);", "alibi"),
+    ("alibi_signed_distance", "bias[cc] = -(double)slopes[h] * fabs((double)pos[r] - (double)pos[kr]);",
+     "bias[cc] = -(double)slopes[h] * ((double)pos[kr] - (double)pos[r]);", "alibi"),
+    ("alibi_decode_tail_position_from_cache", "const double pk = cc < n_cache ? (double)cache_pos[kr] : (double)tail_pos[kr];",
+     "const double pk = (double)cache_pos[kr];", "alibi"),
     ("decode_forgets_tail", "for (int j = 0; j < tl; ++j, ++c) {", "for (int j = 0; j < 0; ++j, ++c) {", "decode"),
     ("decode_keeps_only_first_path", "for (int jj = 0; jj < k; ++jj) {\n                const int i = kept_idx[b * k + jj];\n                if (i < ppo[b] || i >= ppo[b + 1]) continue;",
      "for (int jj = 0; jj < (k > 1 ? 1 : k); ++jj) {\n                const int i = kept_idx[b * k + jj];\n                if (i < ppo[b] || i >= ppo[b + 1]) continue;", "decode"),

@@ -245,6 +245,112 @@ def test_prefill_degenerate_rows():
 
 
 # ---------------------------------------------------------------- O4 path scores
+# ---------------------------------------------------------------------- ALiBi bias (prefill)
+def _alibi_slopes(H):
+    return np.array([2.0 ** (-8.0 * (h + 1) / H) for h in range(H)], np.float32)
+
+
+def test_prefill_alibi_single_path_is_textbook_alibi():
+    """One path, integer positions 0..n-1: causal attention with the additive bias
+    -slope_h * (i - j), checked against torch SDPA given that bias as an explicit mask."""
+    P, L, Q, H, D = 5, 8, 3, 4, 16
+    n = P + L + Q
+    lay = build_layout([P], [[L]], [[Q]])
+    q, k, v = _rand_qkv(n, H, H, D)
+    slopes = _alibi_slopes(H)
+    pos = np.arange(n, dtype=np.float32)
+    out, _ = oracle.prefill(q, k, v, lay, 1 / math.sqrt(D), pos=pos, slopes=slopes)
+    i, j = torch.arange(n)[:, None], torch.arange(n)[None, :]
+    bias = -torch.from_numpy(slopes).double()[:, None, None] * (i - j).double()
+    bias = bias.masked_fill(j > i, float("-inf"))
+    tq, tk, tv = (torch.from_numpy(a).double().permute(1, 0, 2)[None] for a in (q, k, v))
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, attn_mask=bias[None])[0].permute(1, 0, 2)
+    np.testing.assert_allclose(out, ref.numpy(), atol=2e-6)
+
+
+def test_prefill_alibi_fork_join_dense_and_invariances():
+    lay = build_layout([5, 0, 3], [[4, 1, 7], [6, 2], [0, 5]], [[3, 3, 3], [2, 2], [4, 4]])
+    T, H = lay.total_tokens, 4
+    q, k, v = _rand_qkv(T, H, 2, 8)
+    slopes = _alibi_slopes(H)
+    # fractional positions, as the equilibrium assignment produces
+    pos = np.concatenate([oracle.positions(int(lay.pre_len[b]), lay.doc_len[lay.prompt_path_off[b]:lay.prompt_path_off[b + 1]],
+                                           int(lay.qry_len[lay.prompt_path_off[b]]))[0] for b in range(3)]).astype(np.float32)
+    assert pos.shape == (T,) and np.any(pos != np.round(pos))
+    out, lse = oracle.prefill(q, k, v, lay, 0.4, pos=pos, slopes=slopes)
+    mask = _dag_mask(lay)
+    dist = np.abs(pos.astype(np.float64)[:, None] - pos.astype(np.float64)[None, :])
+    for h in range(H):              # dense reference, one head at a time: scores + bias matrix
+        sc = 0.4 * q[:, h].astype(np.float64) @ k[:, h // 2].astype(np.float64).T - float(slopes[h]) * dist
+        sc = np.where(mask, sc, -np.inf)
+        m = sc.max(axis=1, keepdims=True)
+        e = np.exp(sc - m)
+        np.testing.assert_allclose(out[:, h], (e / e.sum(1, keepdims=True)) @ v[:, h // 2].astype(np.float64), atol=2e-6)
+        np.testing.assert_allclose(lse[h], (m + np.log(e.sum(1, keepdims=True)))[:, 0], atol=2e-6)
+    plain, plain_l = oracle.prefill(q, k, v, lay, 0.4)
+    zero, zero_l = oracle.prefill(q, k, v, lay, 0.4, pos=pos, slopes=np.zeros(H, np.float32))
+    np.testing.assert_array_equal(zero, plain)                      # zero slopes: no bias
+    same, _ = oracle.prefill(q, k, v, lay, 0.4, pos=np.full(T, 3.25, np.float32), slopes=slopes)
+    np.testing.assert_allclose(same, plain, atol=1e-6)              # all tokens at one position: no bias
+    shifted, _ = oracle.prefill(q, k, v, lay, 0.4, pos=pos + 64.0, slopes=slopes)
+    np.testing.assert_allclose(shifted, out, atol=1e-5)             # only distances matter
+    assert np.abs(out - plain).max() > 1e-3                         # and the bias does something
+
+
+def test_prefill_alibi_steep_slope_attends_to_itself():
+    """slope -> infinity: every key but the row's own (distance 0) is suppressed, so out = v."""
+    lay = build_layout([3], [[4, 2]], [[2, 2]])
+    T = lay.total_tokens
+    q, k, v = _rand_qkv(T, 2, 2, 8)
+    pos = oracle.positions(3, [4, 2], 2)[0].astype(np.float32)
+    out, _ = oracle.prefill(q, k, v, lay, 0.3, pos=pos, slopes=np.full(2, 1e4, np.float32))
+    np.testing.assert_allclose(out, v, atol=1e-6)
+
+
+def test_decode_alibi_dense_and_matches_prefill_row():
+    lay, H, Hkv, D, q, kc, vc, tk, tv = _decode_setup()
+    slopes = _alibi_slopes(H)
+    cpos = (np.arange(lay.total_tokens) * 0.75 + 1.0).astype(np.float32)
+    tpos = np.array([[40.0, 41.0, 42.0], [30.5, 31.5, 32.5]], np.float32)
+    qpos = np.array([42.0, 30.5], np.float32)
+    kept = np.array([[2, 0], [4, -1]], np.int32)
+    tl = np.array([3, 1], np.int32)
+    out, lse = oracle.pruned_decode(q, kc, vc, lay, kept, tk, tv, tl, 0.35, q_pos=qpos, cache_pos=cpos, tail_pos=tpos, slopes=slopes)
+    for b in range(2):
+        rows = list(range(lay.pre_start[b], lay.pre_start[b] + lay.pre_len[b]))
+        for i in kept[b]:
+            if i >= 0:
+                rows += list(range(lay.path_start[i], lay.path_start[i] + lay.doc_len[i] + lay.qry_len[i]))
+        kpos = np.concatenate([cpos[rows], tpos[b, :tl[b]]]).astype(np.float64)
+        for h in range(H):
+            keys = np.concatenate([kc[rows, h // 2], tk[b, :tl[b], h // 2]]).astype(np.float64)
+            vals = np.concatenate([vc[rows, h // 2], tv[b, :tl[b], h // 2]]).astype(np.float64)
+            sc = 0.35 * keys @ q[b, h].astype(np.float64) - float(slopes[h]) * np.abs(float(qpos[b]) - kpos)
+            e = np.exp(sc - sc.max())
+            np.testing.assert_allclose(out[b, h], (e / e.sum()) @ vals, atol=2e-6)
+            assert lse[b, h] == pytest.approx(sc.max() + math.log(e.sum()), abs=2e-6)
+    plain, _ = oracle.pruned_decode(q, kc, vc, lay, kept, tk, tv, tl, 0.35)
+    zero, _ = oracle.pruned_decode(q, kc, vc, lay, kept, tk, tv, tl, 0.35, q_pos=qpos, cache_pos=cpos, tail_pos=tpos,
+                                   slopes=np.zeros(H, np.float32))
+    np.testing.assert_array_equal(zero, plain)
+    # k = 1: the decoded token is the last row of an ALiBi prefill over p + d_i + q_i + [itself]
+    i = 1
+    P, L, Q = int(lay.pre_len[0]), int(lay.doc_len[i]), int(lay.qry_len[i])
+    o1, _ = oracle.pruned_decode(q, kc, vc, lay, np.array([[i], [-1]], np.int32), tk, tv, np.array([1, 1], np.int32), 0.5,
+                                 q_pos=qpos, cache_pos=cpos, tail_pos=tpos, slopes=slopes)
+    ext = build_layout([P], [[L]], [[Q + 1]])
+    rows = list(range(P)) + list(range(lay.path_start[i], lay.path_start[i] + L + Q))
+    q_ext = np.zeros((ext.total_tokens, H, D), np.float32)
+    q_ext[-1] = q[0]
+    pos_ext = np.concatenate([cpos[rows], [qpos[0]]]).astype(np.float32)
+    tpos1 = tpos.copy(); tpos1[0, 0] = qpos[0]
+    o1, _ = oracle.pruned_decode(q, kc, vc, lay, np.array([[i], [-1]], np.int32), tk, tv, np.array([1, 1], np.int32), 0.5,
+                                 q_pos=qpos, cache_pos=cpos, tail_pos=tpos1, slopes=slopes)
+    o_ext, _ = oracle.prefill(q_ext, np.concatenate([kc[rows], tk[0, :1]]), np.concatenate([vc[rows], tv[0, :1]]), ext, 0.5,
+                              pos=pos_ext, slopes=slopes)
+    np.testing.assert_allclose(o1[0], o_ext[-1], atol=1e-6)
+
+
 def test_path_scores_match_log_softmax_gather():
     V, qlens = 97, [3, 5, 1, 4]
     off = np.concatenate([[0], np.cumsum(qlens)]).astype(np.int32)
