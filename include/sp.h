@@ -179,6 +179,31 @@ int sp_pruned_decode(const void *q, const void *k_cache, const void *v_cache,
                      void *stream);
 
 /*
+ * ALiBi variants (Section 3.2.2: the equilibrium assignment yields real-valued positions, which
+ * the ALiBi encoding takes as they are; Section 3.2.1: with ALiBi, position gaps turn into
+ * attention penalties, which is what the equilibrium assignment avoids).  They compute what
+ * sp_superpose_prefill / sp_pruned_decode compute with the additive bias
+ *   -slopes[h] * |pos(query) - pos(key)|
+ * on every admitted score before the softmax.  pos: fp32 [T], the position of every packed
+ * row (sp_positions per prompt); slopes: fp32 [n_heads], >= 0.  For the decode step:
+ * q_pos fp32 [B] (the new token's position), cache_pos fp32 [T] (positions of the cache
+ * rows), tail_pos fp32 [B, tail_cap] (positions of the tail rows; nullable when tail_cap == 0).
+ * All other arguments, workspaces, layouts and error codes are those of the plain entry
+ * points; Q and K are used as given (no rotary embedding is implied).
+ */
+int sp_superpose_prefill_alibi(const void *q, const void *k, const void *v, const sp_layout *lay,
+                               const float *pos, const float *slopes, int n_heads, int n_kv_heads,
+                               int head_dim, float scale, int rows, void *out, float *lse, void *ws,
+                               size_t ws_bytes, int dtype, void *stream);
+int sp_pruned_decode_alibi(const void *q, const void *k_cache, const void *v_cache,
+                           const sp_layout *lay, const int32_t *kept_idx, int k,
+                           const void *tail_k, const void *tail_v, const int32_t *tail_len,
+                           int tail_cap, int64_t max_keys, const float *q_pos, const float *cache_pos,
+                           const float *tail_pos, const float *slopes, int n_heads, int n_kv_heads,
+                           int head_dim, float scale, void *out, float *lse, void *ws, size_t ws_bytes,
+                           int dtype, void *stream);
+
+/*
  * Decode attention without a caller workspace.  (The paper has no counterpart: this entry
  * point exists for integration reasons only.)  It computes exactly what sp_pruned_decode
  * computes, with the same arguments minus (ws, ws_bytes), for callers that are not able to

@@ -29,6 +29,7 @@ EXPORTS = (
     "sp_path_scores_workspace_bytes", "sp_path_scores", "sp_prune_topk",
     "sp_decode_workspace_bytes", "sp_pruned_decode", "sp_check_status",
     "sp_pruned_decode_static_max_bytes", "sp_pruned_decode_static",
+    "sp_superpose_prefill_alibi", "sp_pruned_decode_alibi",
 )
 
 
@@ -77,6 +78,10 @@ def _load() -> ctypes.CDLL:
     lib.sp_pruned_decode_static_max_bytes.restype = sz
     lib.sp_pruned_decode_static.argtypes = [vp, vp, vp, lp, vp, c_int, vp, vp, vp, c_int, c_i64, c_int, c_int, c_int,
                                             c_f, vp, vp, c_int, vp]
+    lib.sp_superpose_prefill_alibi.argtypes = [vp, vp, vp, lp, vp, vp, c_int, c_int, c_int, c_f, c_int, vp, vp, vp, sz,
+                                               c_int, vp]
+    lib.sp_pruned_decode_alibi.argtypes = [vp, vp, vp, lp, vp, c_int, vp, vp, vp, c_int, c_i64, vp, vp, vp, vp, c_int,
+                                           c_int, c_int, c_f, vp, vp, vp, sz, c_int, vp]
     for name in EXPORTS:
         getattr(lib, name)          # raises AttributeError if a declared symbol is not exported
     return lib
@@ -179,6 +184,16 @@ def sp_superpose_prefill(q, k, v, lay: DeviceLayout, scale: float, out, lse=None
                                     _ptr(out), _ptr(lse), _ptr(ws), _nbytes(ws), dtype_code(q), _stream(stream)))
 
 
+def sp_superpose_prefill_alibi(q, k, v, lay: DeviceLayout, pos, slopes, scale: float, out, lse=None, ws=None,
+                               rows: int = SP_ROWS_ALL, stream=None):
+    """sp_superpose_prefill with the ALiBi bias -slopes[h] * |pos[q] - pos[k]| (pos fp32 [T], slopes fp32 [H])."""
+    T, H, D = q.shape
+    Hkv = k.shape[1]
+    _check(lib.sp_superpose_prefill_alibi(_ptr(q), _ptr(k), _ptr(v), ctypes.byref(lay.c), _ptr(pos), _ptr(slopes), H,
+                                          Hkv, D, scale, rows, _ptr(out), _ptr(lse), _ptr(ws), _nbytes(ws),
+                                          dtype_code(q), _stream(stream)))
+
+
 def sp_path_scores_workspace_bytes(n_rows: int) -> int:
     return int(lib.sp_path_scores_workspace_bytes(n_rows))
 
@@ -207,6 +222,19 @@ def sp_pruned_decode(q, k_cache, v_cache, lay: DeviceLayout, kept_idx, k: int, t
     _check(lib.sp_pruned_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), ctypes.byref(lay.c), _ptr(kept_idx), k,
                                 _ptr(tail_k), _ptr(tail_v), _ptr(tail_len), tail_cap, max_keys, H, Hkv, D, scale,
                                 _ptr(out), _ptr(lse), _ptr(ws), _nbytes(ws), dtype_code(q), _stream(stream)))
+
+
+def sp_pruned_decode_alibi(q, k_cache, v_cache, lay: DeviceLayout, kept_idx, k: int, tail_k, tail_v, tail_len,
+                           tail_cap: int, q_pos, cache_pos, tail_pos, slopes, scale: float, out, lse=None, ws=None,
+                           max_keys: int = 0, stream=None):
+    """sp_pruned_decode with the ALiBi bias: q_pos fp32 [B], cache_pos fp32 [T], tail_pos fp32 [B, tail_cap],
+    slopes fp32 [H]."""
+    B, H, D = q.shape
+    Hkv = k_cache.shape[1]
+    _check(lib.sp_pruned_decode_alibi(_ptr(q), _ptr(k_cache), _ptr(v_cache), ctypes.byref(lay.c), _ptr(kept_idx), k,
+                                      _ptr(tail_k), _ptr(tail_v), _ptr(tail_len), tail_cap, max_keys, _ptr(q_pos),
+                                      _ptr(cache_pos), _ptr(tail_pos), _ptr(slopes), H, Hkv, D, scale, _ptr(out),
+                                      _ptr(lse), _ptr(ws), _nbytes(ws), dtype_code(q), _stream(stream)))
 
 
 def sp_pruned_decode_static_max_bytes() -> int:

@@ -34,6 +34,9 @@ struct DecodeArgs {
     unsigned int *counters;  // [B*H], zero on entry
     int k, tail_cap, n_heads, n_kv_heads, n_splits;
     float scale_log2e;
+    // ALiBi variant only: positions of the query token [B], of the cache rows [T] and of the
+    // tail rows [B, tail_cap], and the per-head slopes [H]
+    const float *q_pos, *cache_pos, *tail_pos, *slopes;
 };
 
 // Workspace layout: [0,256) status word | counters [B*H] u32 | partials.
@@ -69,7 +72,9 @@ template <> struct Raw16<float> {
     }
 };
 
-template <typename T, int D>
+// ALIBI: scores get -slope_h * |pos_q - pos_k| (Section 3.2.2: real-valued positions pose no
+// problem for ALiBi); the plain instantiation carries none of that code.
+template <typename T, int D, bool ALIBI>
 __global__ void __launch_bounds__(kDecThreads, 8)
 decode_kernel(const __grid_constant__ DecodeArgs a)
 {
@@ -85,6 +90,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a)
     const T **seg_k = reinterpret_cast<const T **>(smem_raw + round_up((n_seg + 1) * sizeof(int), 16));
     const T **seg_v = seg_k + n_seg;
     float *red = reinterpret_cast<float *>(seg_v + n_seg);                  // [G][D+2]
+    const float **seg_pos = reinterpret_cast<const float **>(red + G * (D + 2));   // [n_seg], ALiBi only
     __shared__ unsigned int s_ticket;
 
     const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -112,6 +118,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a)
         }
         seg_k[sgm] = kc + row * row_elems;
         seg_v[sgm] = vc + row * row_elems;
+        if (ALIBI) seg_pos[sgm] = (sgm == a.k + 1 && len ? a.tail_pos : a.cache_pos) + row;
         seg_lo[sgm + 1] = len;
     }
     __syncthreads();
@@ -135,10 +142,13 @@ decode_kernel(const __grid_constant__ DecodeArgs a)
     float m = -INFINITY, l = 0.f, acc[N];
 #pragma unroll
     for (int e = 0; e < N; ++e) acc[e] = 0.f;
+    const float q_pos = ALIBI ? a.q_pos[b] : 0.f;
+    const float slope_l2 = ALIBI ? a.slopes[h] * kLog2eD : 0.f;
 
     int seg = 0;
     for (int base = lo; base < hi; base += G * kDecUnroll) {   // trip count is block-uniform
         uint4 kr[kDecUnroll], vr[kDecUnroll];
+        float kpos[kDecUnroll];
         bool live[kDecUnroll];
 #pragma unroll
         for (int u = 0; u < kDecUnroll; ++u) {                  // all loads of the batch first
@@ -149,6 +159,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a)
                 const int64_t off = (int64_t)(j - seg_lo[seg]) * row_elems + sub * N;
                 kr[u] = ld_stream16(seg_k[seg] + off);
                 vr[u] = ld_stream16(seg_v[seg] + off);
+                if (ALIBI) kpos[u] = seg_pos[seg][j - seg_lo[seg]];
             }
         }
         float s[kDecUnroll], cm = -INFINITY;
@@ -163,6 +174,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a)
             }
 #pragma unroll
             for (int o = LPK / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+            if (ALIBI && live[u]) d -= slope_l2 * fabsf(q_pos - kpos[u]);
             s[u] = live[u] ? d : -INFINITY;
             cm = fmaxf(cm, s[u]);
         }
@@ -245,20 +257,25 @@ decode_kernel(const __grid_constant__ DecodeArgs a)
     }
 }
 
-template <typename T, int D>
-static int launch_decode(const DecodeArgs &a, int n_prompts, cudaStream_t st)
+template <typename T, int D, bool ALIBI>
+static int launch_decode_v(const DecodeArgs &a, int n_prompts, cudaStream_t st)
 {
     constexpr int G = kDecThreads / (D / Vec<T>::N);
     const int n_seg = a.k + 2;
     const size_t smem = round_up((n_seg + 1) * sizeof(int), 16) + 2 * n_seg * sizeof(void *) +
-                        (size_t)G * (D + 2) * sizeof(float);
+                        (size_t)G * (D + 2) * sizeof(float) + (ALIBI ? n_seg * sizeof(void *) : 0);
     SP_REQUIRE(smem <= 200 * 1024, SP_ERR_UNSUPPORTED, "sp_pruned_decode: k = %d needs too much shared memory", a.k);
     if (smem > 48 * 1024)
-        SP_CUDA(cudaFuncSetAttribute(decode_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        SP_CUDA(cudaFuncSetAttribute(decode_kernel<T, D, ALIBI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     dim3 grid(a.n_splits, a.n_heads, n_prompts);
-    decode_kernel<T, D><<<grid, kDecThreads, smem, st>>>(a);
+    decode_kernel<T, D, ALIBI><<<grid, kDecThreads, smem, st>>>(a);
     SP_CUDA(cudaGetLastError());
     return SP_OK;
+}
+template <typename T, int D>
+static int launch_decode(const DecodeArgs &a, int n_prompts, cudaStream_t st)
+{
+    return a.slopes ? launch_decode_v<T, D, true>(a, n_prompts, st) : launch_decode_v<T, D, false>(a, n_prompts, st);
 }
 
 }  // namespace sp
@@ -272,14 +289,15 @@ extern "C" size_t sp_decode_workspace_bytes(int n_prompts, int n_heads, int head
     return 256 + decode_counter_bytes(n_prompts, n_heads) + round_up(part, 256);
 }
 
-extern "C" int sp_pruned_decode(const void *q, const void *k_cache, const void *v_cache,
-                                const sp_layout *lay, const int32_t *kept_idx, int k,
-                                const void *tail_k, const void *tail_v, const int32_t *tail_len,
-                                int tail_cap, int64_t max_keys, int n_heads, int n_kv_heads,
-                                int head_dim, float scale, void *out, float *lse, void *ws,
-                                size_t ws_bytes, int dtype, void *stream)
+namespace sp {
+static int decode_with_workspace(const void *q, const void *k_cache, const void *v_cache,
+                                 const sp_layout *lay, const int32_t *kept_idx, int k,
+                                 const void *tail_k, const void *tail_v, const int32_t *tail_len,
+                                 int tail_cap, int64_t max_keys, const float *q_pos, const float *cache_pos,
+                                 const float *tail_pos, const float *slopes, int n_heads, int n_kv_heads,
+                                 int head_dim, float scale, void *out, float *lse, void *ws,
+                                 size_t ws_bytes, int dtype, void *stream)
 {
-    using namespace sp;
     SP_REQUIRE(dtype == SP_F32 || dtype == SP_BF16, SP_ERR_INVALID_ARG, "sp_pruned_decode: unknown dtype %d", dtype);
     if (int rc = check_layout(lay)) return rc;
     SP_REQUIRE(head_dim == 64 || head_dim == 128, SP_ERR_UNSUPPORTED, "sp_pruned_decode: head_dim %d (64 or 128 supported)", head_dim);
@@ -318,12 +336,42 @@ extern "C" int sp_pruned_decode(const void *q, const void *k_cache, const void *
     a.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + 256 + cbytes);
     a.k = k; a.tail_cap = tail_cap; a.n_heads = n_heads; a.n_kv_heads = n_kv_heads;
     a.n_splits = n_splits; a.scale_log2e = scale * kLog2eD;
+    a.q_pos = q_pos; a.cache_pos = cache_pos; a.tail_pos = tail_pos; a.slopes = slopes;
 
     if (dtype == SP_BF16)
         return head_dim == 128 ? launch_decode<__nv_bfloat16, 128>(a, lay->n_prompts, st)
                                : launch_decode<__nv_bfloat16, 64>(a, lay->n_prompts, st);
     return head_dim == 128 ? launch_decode<float, 128>(a, lay->n_prompts, st)
                            : launch_decode<float, 64>(a, lay->n_prompts, st);
+}
+}  // namespace sp
+
+extern "C" int sp_pruned_decode(const void *q, const void *k_cache, const void *v_cache,
+                                const sp_layout *lay, const int32_t *kept_idx, int k,
+                                const void *tail_k, const void *tail_v, const int32_t *tail_len,
+                                int tail_cap, int64_t max_keys, int n_heads, int n_kv_heads,
+                                int head_dim, float scale, void *out, float *lse, void *ws,
+                                size_t ws_bytes, int dtype, void *stream)
+{
+    return sp::decode_with_workspace(q, k_cache, v_cache, lay, kept_idx, k, tail_k, tail_v, tail_len, tail_cap,
+                                     max_keys, nullptr, nullptr, nullptr, nullptr, n_heads, n_kv_heads, head_dim,
+                                     scale, out, lse, ws, ws_bytes, dtype, stream);
+}
+
+extern "C" int sp_pruned_decode_alibi(const void *q, const void *k_cache, const void *v_cache,
+                                      const sp_layout *lay, const int32_t *kept_idx, int k,
+                                      const void *tail_k, const void *tail_v, const int32_t *tail_len,
+                                      int tail_cap, int64_t max_keys, const float *q_pos,
+                                      const float *cache_pos, const float *tail_pos, const float *slopes,
+                                      int n_heads, int n_kv_heads, int head_dim, float scale, void *out,
+                                      float *lse, void *ws, size_t ws_bytes, int dtype, void *stream)
+{
+    using namespace sp;
+    SP_REQUIRE(lay == nullptr || lay->n_prompts == 0 || (q_pos && cache_pos && slopes && (tail_cap == 0 || tail_pos)),
+               SP_ERR_INVALID_ARG, "sp_pruned_decode_alibi: q_pos, cache_pos, slopes (and tail_pos with a tail) are required");
+    return decode_with_workspace(q, k_cache, v_cache, lay, kept_idx, k, tail_k, tail_v, tail_len, tail_cap, max_keys,
+                                 q_pos, cache_pos, tail_pos, slopes, n_heads, n_kv_heads, head_dim, scale, out,
+                                 lse, ws, ws_bytes, dtype, stream);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -415,6 +463,7 @@ extern "C" int sp_pruned_decode_static(const void *q, const void *k_cache, const
     a.partial = reinterpret_cast<float *>(scratch + cbytes);
     a.k = k; a.tail_cap = tail_cap; a.n_heads = n_heads; a.n_kv_heads = n_kv_heads;
     a.n_splits = n_splits; a.scale_log2e = scale * kLog2eD;
+    a.q_pos = nullptr; a.cache_pos = nullptr; a.tail_pos = nullptr; a.slopes = nullptr;
 
     if (dtype == SP_BF16)
         return head_dim == 128 ? launch_decode<__nv_bfloat16, 128>(a, lay->n_prompts, st)

@@ -4,16 +4,17 @@
 #include "common.cuh"
 
 namespace sp {
-int launch_prefill_simt(const void *q, const void *k, const void *v, const sp_layout *lay, int n_heads,
-                        int n_kv_heads, int head_dim, float scale, int rows, void *out, float *lse,
-                        int dtype, cudaStream_t st);
+int launch_prefill_simt(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos,
+                        const float *slopes, int n_heads, int n_kv_heads, int head_dim, float scale, int rows,
+                        void *out, float *lse, int dtype, cudaStream_t st);
 size_t prefill_tc_workspace_bytes(int n_prompts, int n_paths, int max_pre_len, int max_path_len, int n_heads);
-int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layout *lay, int n_heads,
-                      int n_kv_heads, float scale, int rows, void *out, float *lse, void *ws,
-                      size_t ws_bytes, cudaStream_t st);
+int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos,
+                      const float *slopes, int n_heads, int n_kv_heads, float scale, int rows, void *out,
+                      float *lse, void *ws, size_t ws_bytes, cudaStream_t st);
 size_t prefill_qonly_workspace_bytes(int n_prompts, int n_paths, int max_pre_len, int max_path_len);
-int launch_prefill_qonly(const void *q, const void *k, const void *v, const sp_layout *lay, int n_heads,
-                         int n_kv_heads, float scale, void *out, float *lse, void *ws, cudaStream_t st);
+int launch_prefill_qonly(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos,
+                         const float *slopes, int n_heads, int n_kv_heads, float scale, void *out, float *lse,
+                         void *ws, cudaStream_t st);
 }  // namespace sp
 
 extern "C" size_t sp_prefill_workspace_bytes(int n_prompts, int n_paths, int max_pre_len,
@@ -25,12 +26,11 @@ extern "C" size_t sp_prefill_workspace_bytes(int n_prompts, int n_paths, int max
     return 256;
 }
 
-extern "C" int sp_superpose_prefill(const void *q, const void *k, const void *v, const sp_layout *lay,
-                                    int n_heads, int n_kv_heads, int head_dim, float scale, int rows,
-                                    void *out, float *lse, void *ws, size_t ws_bytes, int dtype,
-                                    void *stream)
+namespace sp {
+static int prefill_entry(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos,
+                         const float *slopes, int n_heads, int n_kv_heads, int head_dim, float scale, int rows,
+                         void *out, float *lse, void *ws, size_t ws_bytes, int dtype, void *stream)
 {
-    using namespace sp;
     SP_REQUIRE(dtype == SP_F32 || dtype == SP_BF16, SP_ERR_INVALID_ARG, "sp_superpose_prefill: unknown dtype %d", dtype);
     if (int rc = check_layout(lay)) return rc;
     SP_REQUIRE(head_dim == 64 || head_dim == 128, SP_ERR_UNSUPPORTED,
@@ -51,9 +51,31 @@ extern "C" int sp_superpose_prefill(const void *q, const void *k, const void *v,
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (dtype == SP_BF16 && head_dim == 128 && rows == SP_ROWS_QUERY_ONLY)
-        return launch_prefill_qonly(q, k, v, lay, n_heads, n_kv_heads, scale, out, lse, ws, st);
+        return launch_prefill_qonly(q, k, v, lay, pos, slopes, n_heads, n_kv_heads, scale, out, lse, ws, st);
     if (dtype == SP_BF16 && head_dim == 128)
-        return launch_prefill_tc(q, k, v, lay, n_heads, n_kv_heads, scale, rows, out, lse, ws, ws_bytes, st);
+        return launch_prefill_tc(q, k, v, lay, pos, slopes, n_heads, n_kv_heads, scale, rows, out, lse, ws, ws_bytes, st);
     SP_CUDA(cudaMemsetAsync(ws, 0, 256, st));
-    return launch_prefill_simt(q, k, v, lay, n_heads, n_kv_heads, head_dim, scale, rows, out, lse, dtype, st);
+    return launch_prefill_simt(q, k, v, lay, pos, slopes, n_heads, n_kv_heads, head_dim, scale, rows, out, lse, dtype, st);
+}
+}  // namespace sp
+
+extern "C" int sp_superpose_prefill(const void *q, const void *k, const void *v, const sp_layout *lay,
+                                    int n_heads, int n_kv_heads, int head_dim, float scale, int rows,
+                                    void *out, float *lse, void *ws, size_t ws_bytes, int dtype,
+                                    void *stream)
+{
+    return sp::prefill_entry(q, k, v, lay, nullptr, nullptr, n_heads, n_kv_heads, head_dim, scale, rows, out, lse,
+                             ws, ws_bytes, dtype, stream);
+}
+
+extern "C" int sp_superpose_prefill_alibi(const void *q, const void *k, const void *v, const sp_layout *lay,
+                                          const float *pos, const float *slopes, int n_heads, int n_kv_heads,
+                                          int head_dim, float scale, int rows, void *out, float *lse, void *ws,
+                                          size_t ws_bytes, int dtype, void *stream)
+{
+    using namespace sp;
+    SP_REQUIRE(lay == nullptr || lay->total_tokens == 0 || (pos && slopes), SP_ERR_INVALID_ARG,
+               "sp_superpose_prefill_alibi: pos and slopes are required");
+    return prefill_entry(q, k, v, lay, pos, slopes, n_heads, n_kv_heads, head_dim, scale, rows, out, lse, ws,
+                         ws_bytes, dtype, stream);
 }

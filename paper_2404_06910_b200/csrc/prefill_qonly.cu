@@ -36,6 +36,7 @@ struct QoParams {
     int n_heads, n_kv_heads, kv_group;
     int64_t total_tokens;
     float scale_log2e;
+    const float *pos, *slopes;       // ALiBi variant: token positions [T], head slopes [H]
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -144,6 +145,8 @@ __device__ __forceinline__ void load_rows(unsigned char *dst, const unsigned cha
     }
 }
 
+// ALIBI: scores get -slope_h * |pos_q - pos_k| before the softmax (Section 3.2.2).
+template <bool ALIBI>
 __global__ void __launch_bounds__(kQThreads, kQBlocksPerSM) prefill_qonly_kernel(const QoParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -183,6 +186,7 @@ __global__ void __launch_bounds__(kQThreads, kQBlocksPerSM) prefill_qonly_kernel
     uint32_t qf[kQD / 16][4];        // this warp's 16 query rows as A fragments
     float o[kQD / 8][4];             // O accumulator: 16 rows x 128 columns
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // rows gid and gid + 8
+    float pq[2] = {0.f, 0.f}, slope_l2 = 0.f;                         // ALiBi: the two rows' positions
 
     while (cc.valid) {
         // tile cc.g must have landed: all groups but the ones of the tiles fetched after it
@@ -197,6 +201,14 @@ __global__ void __launch_bounds__(kQThreads, kQBlocksPerSM) prefill_qonly_kernel
 #pragma unroll
             for (int i = 0; i < kQD / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
             m_run[0] = m_run[1] = -INFINITY; l_run[0] = l_run[1] = 0.f;
+            if (ALIBI) {
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int rowq = warp * 16 + gid + 8 * hh;
+                    pq[hh] = rowq < cc.t.n_rows ? p.pos[cc.t.q_row + rowq] : 0.f;
+                }
+                slope_l2 = p.slopes[cc.h] * kLog2eQ;
+            }
             __syncthreads();         // both warps hold their Q before the next item's may be fetched
             q_held = (int)cc.item_no;
         }
@@ -223,6 +235,16 @@ __global__ void __launch_bounds__(kQThreads, kQBlocksPerSM) prefill_qonly_kernel
 
         // ---- online softmax (log2 units); keys past a row's limit count as -inf
         uint32_t pa[kQN / 16][4];
+        float pk[kQN / 8][2];        // ALiBi: positions of this thread's eight key columns
+        if (ALIBI) {
+#pragma unroll
+            for (int nt = 0; nt < kQN / 8; ++nt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int col = nt * 8 + 2 * tig + e;
+                    pk[nt][e] = col < kt.n_valid ? p.pos[kt.row0 + col] : 0.f;
+                }
+        }
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
             const int rowq = warp * 16 + gid + 8 * hh;
@@ -233,7 +255,9 @@ __global__ void __launch_bounds__(kQThreads, kQBlocksPerSM) prefill_qonly_kernel
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const int col = nt * 8 + 2 * tig + e;
-                    const float x = col < lim ? s[nt][2 * hh + e] * p.scale_log2e : -INFINITY;
+                    float x = s[nt][2 * hh + e] * p.scale_log2e;
+                    if (ALIBI) x -= slope_l2 * fabsf(pq[hh] - pk[nt][e]);
+                    x = col < lim ? x : -INFINITY;
                     s[nt][2 * hh + e] = x;
                     mx = fmaxf(mx, x);
                 }
@@ -310,8 +334,9 @@ size_t prefill_qonly_workspace_bytes(int n_prompts, int n_paths, int max_pre_len
     return 256 + round_up((size_t)plan_max_tiles(0, n_paths, 0, max_path_len, kQM) * sizeof(TcTile), 256);
 }
 
-int launch_prefill_qonly(const void *q, const void *k, const void *v, const sp_layout *lay, int n_heads,
-                         int n_kv_heads, float scale, void *out, float *lse, void *ws, cudaStream_t st)
+int launch_prefill_qonly(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos,
+                         const float *slopes, int n_heads, int n_kv_heads, float scale, void *out, float *lse,
+                         void *ws, cudaStream_t st)
 {
     TcHeader *hdr = static_cast<TcHeader *>(ws);
     TcTile *tiles = reinterpret_cast<TcTile *>(static_cast<char *>(ws) + 256);
@@ -333,10 +358,16 @@ int launch_prefill_qonly(const void *q, const void *k, const void *v, const sp_l
     p.hdr = hdr; p.tiles = tiles;
     p.n_heads = n_heads; p.n_kv_heads = n_kv_heads; p.kv_group = n_heads / n_kv_heads;
     p.total_tokens = lay->total_tokens; p.scale_log2e = scale * kLog2eQ;
+    p.pos = pos; p.slopes = slopes;
     const int smem = (2 * kQStages + 1) * kTileB;
-    SP_CUDA(cudaFuncSetAttribute(prefill_qonly_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int grid = (int)std::min<int64_t>(items, (int64_t)kQBlocksPerSM * kNumSMs);
-    prefill_qonly_kernel<<<grid, kQThreads, smem, st>>>(p);
+    if (pos) {
+        SP_CUDA(cudaFuncSetAttribute(prefill_qonly_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        prefill_qonly_kernel<true><<<grid, kQThreads, smem, st>>>(p);
+    } else {
+        SP_CUDA(cudaFuncSetAttribute(prefill_qonly_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        prefill_qonly_kernel<false><<<grid, kQThreads, smem, st>>>(p);
+    }
     SP_CUDA(cudaGetLastError());
     return SP_OK;
 }

@@ -22,6 +22,7 @@ struct PrefillSimtArgs {
     int n_prompts, n_paths, n_heads, n_kv_heads, rows_mode;
     int64_t total_tokens;
     float scale_log2e;
+    const float *pos, *slopes;   // ALiBi: token positions [T] and head slopes [H]; NULL = no bias
 };
 
 template <typename T, int EPL> struct LaneVec;     // EPL contiguous elements of one lane
@@ -82,6 +83,8 @@ prefill_simt_kernel(const __grid_constant__ PrefillSimtArgs a)
 #pragma unroll
         for (int e = 0; e < EPL; ++e) { qf[e] *= a.scale_log2e; acc[e] = 0.f; }
         float m = -INFINITY, l = 0.f;
+        const float pq = a.pos ? a.pos[r] : 0.f;
+        const float slope_l2 = a.pos ? a.slopes[h] * kLog2eP : 0.f;
 
         const int n_keys = pre_n + j + 1;
         for (int c = 0; c < n_keys; ++c) {
@@ -93,6 +96,7 @@ prefill_simt_kernel(const __grid_constant__ PrefillSimtArgs a)
 #pragma unroll
             for (int e = 0; e < EPL; ++e) s = fmaf(qf[e], kf[e], s);
             s = warp_sum(s);
+            if (a.pos) s -= slope_l2 * fabsf(pq - a.pos[kr]);     // ALiBi: linear distance penalty
             if (s > m) {
                 const float rs = exp2f(m - s);
                 l *= rs;
@@ -113,9 +117,9 @@ prefill_simt_kernel(const __grid_constant__ PrefillSimtArgs a)
     }
 }
 
-int launch_prefill_simt(const void *q, const void *k, const void *v, const sp_layout *lay, int n_heads,
-                        int n_kv_heads, int head_dim, float scale, int rows, void *out, float *lse,
-                        int dtype, cudaStream_t st)
+int launch_prefill_simt(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos,
+                        const float *slopes, int n_heads, int n_kv_heads, int head_dim, float scale, int rows,
+                        void *out, float *lse, int dtype, cudaStream_t st)
 {
     PrefillSimtArgs a;
     a.q = q; a.k = k; a.v = v; a.out = out; a.lse = lse;
@@ -123,6 +127,7 @@ int launch_prefill_simt(const void *q, const void *k, const void *v, const sp_la
     a.path_start = lay->path_start; a.doc_len = lay->doc_len; a.qry_len = lay->qry_len;
     a.n_prompts = lay->n_prompts; a.n_paths = lay->n_paths; a.n_heads = n_heads; a.n_kv_heads = n_kv_heads;
     a.rows_mode = rows; a.total_tokens = lay->total_tokens; a.scale_log2e = scale * kLog2eP;
+    a.pos = pos; a.slopes = slopes;
     const dim3 grid(lay->n_prompts + lay->n_paths, n_heads);
     const int threads = kSimtWarps * 32;
     if (dtype == SP_F32) {

@@ -62,6 +62,7 @@ struct TcParams {
     int n_heads, kv_group;
     int64_t total_tokens;
     float scale_log2e;
+    const float *pos, *slopes;        // ALiBi variant: token positions [T], head slopes [H]
     int stall_producer;               // test hook: the producer issues no load, so every wait runs out
 };
 
@@ -142,6 +143,9 @@ enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_V_FULL = BAR_K_FULL + 2, BAR
 template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
+// ALIBI: scores get -slope_h * |pos_q - pos_k| before the softmax (Section 3.2.2: real-valued
+// positions are no obstacle for ALiBi); the plain instantiation carries none of that code.
+template <bool ALIBI>
 __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_constant__ TcParams p)
 {
     extern __shared__ unsigned char smem_raw[];
@@ -288,6 +292,8 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
         Cursor c;
         c.init(p.tiles, n_items, p.n_heads);
         float m_ref = -INFINITY, l = 0.f;          // reference maximum (log2 units) and row sum
+        float pq = 0.f, slope_l2 = 0.f;            // ALiBi: this row's position, the head's slope (log2 units)
+        const float sc_exp = ALIBI ? 1.f : sc;     // ALiBi scores are scaled when the bias is added
 
         while (c.valid && ok) {
             const int st = c.g & 1;
@@ -305,7 +311,13 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             const bool live_w = warp * 32 < t.n_rows;
             const bool use0 = live_w && lim31 > 0;               // uniform: keys [0,32) seen by some row
             const bool use1 = live_w && lim31 > 32;              // uniform: keys [32,64) seen by some row
-            if (first) { m_ref = -INFINITY; l = 0.f; }
+            if (first) {
+                m_ref = -INFINITY; l = 0.f;
+                if (ALIBI) {
+                    pq = row < t.n_rows ? p.pos[t.q_row + row] : 0.f;
+                    slope_l2 = p.slopes[c.h] * kLog2eT;
+                }
+            }
             if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
             tc_fence_after();
 
@@ -316,6 +328,22 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             // keys past the row's limit (causal diagonal, ragged tail) -> -inf; skipped when the
             // whole warp sees everything it loaded
             float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            if (ALIBI) {                // score * scale - slope * |distance|, every thread reads the same key positions
+                if (use0) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float pk = i < kt.n_valid ? __ldg(p.pos + kt.row0 + i) : 0.f;
+                        r0[i] = __float_as_uint(fmaf(__uint_as_float(r0[i]), sc, -slope_l2 * fabsf(pq - pk)));
+                    }
+                }
+                if (use1) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float pk = 32 + i < kt.n_valid ? __ldg(p.pos + kt.row0 + 32 + i) : 0.f;
+                        r1[i] = __float_as_uint(fmaf(__uint_as_float(r1[i]), sc, -slope_l2 * fabsf(pq - pk)));
+                    }
+                }
+            }
             if (use0) {
                 if (lim0 < 32) {
 #pragma unroll
@@ -332,7 +360,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
 #pragma unroll
                 for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(r1[i]));
             }
-            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;
+            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc_exp;
             float alpha = 1.f;
             bool grow = false;
             if (first) {
@@ -367,8 +395,8 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                         uint32_t pk[8];
 #pragma unroll
                         for (int i = 0; i < 16; i += 2) {
-                            const float p0 = ex2(fmaf(__uint_as_float(r0[q8 * 16 + i]), sc, nm));
-                            const float p1 = ex2(fmaf(__uint_as_float(r0[q8 * 16 + i + 1]), sc, nm));
+                            const float p0 = ex2(fmaf(__uint_as_float(r0[q8 * 16 + i]), sc_exp, nm));
+                            const float p1 = ex2(fmaf(__uint_as_float(r0[q8 * 16 + i + 1]), sc_exp, nm));
                             rs[(i >> 1) & 3] += p0 + p1;
                             pk[i >> 1] = pack_bf16x2(p0, p1);
                         }
@@ -388,8 +416,8 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                             uint32_t pk[8];
 #pragma unroll
                             for (int i = 0; i < 16; i += 2) {
-                                const float p0 = ex2(fmaf(__uint_as_float(r1[q8 * 16 + i]), sc, nm));
-                                const float p1 = ex2(fmaf(__uint_as_float(r1[q8 * 16 + i + 1]), sc, nm));
+                                const float p0 = ex2(fmaf(__uint_as_float(r1[q8 * 16 + i]), sc_exp, nm));
+                                const float p1 = ex2(fmaf(__uint_as_float(r1[q8 * 16 + i + 1]), sc_exp, nm));
                                 rs[(i >> 1) & 3] += p0 + p1;
                                 pk[i >> 1] = pack_bf16x2(p0, p1);
                             }
@@ -521,9 +549,9 @@ size_t prefill_tc_workspace_bytes(int n_prompts, int n_paths, int max_pre_len, i
     return 256 + round_up((size_t)max_tiles(n_prompts, n_paths, max_pre_len, max_path_len) * sizeof(TcTile), 256);
 }
 
-int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layout *lay, int n_heads,
-                      int n_kv_heads, float scale, int rows, void *out, float *lse, void *ws,
-                      size_t, cudaStream_t st)
+int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos,
+                      const float *slopes, int n_heads, int n_kv_heads, float scale, int rows, void *out,
+                      float *lse, void *ws, size_t, cudaStream_t st)
 {
     static EncodeTiledFn enc = nullptr;
     if (!enc) {
@@ -560,6 +588,7 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
     p.out = static_cast<__nv_bfloat16 *>(out); p.lse = lse;
     p.n_heads = n_heads; p.kv_group = n_heads / n_kv_heads;
     p.total_tokens = lay->total_tokens; p.scale_log2e = scale * kLog2eT;
+    p.pos = pos; p.slopes = slopes;
     // Failure-detection test hook (host-injected, no GPU fault): with SP_TEST_STALL_PRODUCER=1 in
     // the environment no tile is ever loaded, every bounded wait expires, the blocks unwind and
     // the call reports SP_ERR_TIMEOUT through the workspace status word.
@@ -570,8 +599,13 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
     if (items == 0) return SP_OK;
     const int grid = (int)std::min<int64_t>(items, 2 * kNumSMs);
     const int smem = kQBytes + 4 * kKVBytes + 4 * 2048 + 1024;
-    SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    prefill_tc_kernel<<<grid, kTcThreads, smem, st>>>(p);
+    if (pos) {
+        SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        prefill_tc_kernel<true><<<grid, kTcThreads, smem, st>>>(p);
+    } else {
+        SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        prefill_tc_kernel<false><<<grid, kTcThreads, smem, st>>>(p);
+    }
     SP_CUDA(cudaGetLastError());
     return SP_OK;
 }

@@ -566,3 +566,71 @@ def test_iterative_superposition_rounds():
                         workspace(sp.sp_decode_workspace_bytes(B, H, D)))
     ref_d, _ = oracle.pruned_decode(f32(dq), k_r, f32(v), lay, ref_kept, f32(tk), f32(tv), tl, scale)
     assert rel_l2(f32(o), ref_d) <= TOL["bf16"]
+
+
+# ------------------------------------------------------------------------- ALiBi variants
+def _slopes(H):
+    return np.array([2.0 ** (-8.0 * (h + 1) / H) for h in range(H)], np.float32)
+
+
+@pytest.mark.parametrize("dtype,D,rows", [("f32", 64, "all"), ("bf16", 64, "all"), ("bf16", 128, "all"), ("bf16", 128, "query"),
+                                          ("f32", 128, "query")])
+def test_prefill_alibi_parity(dtype, D, rows):
+    """Fork-join prefill with the ALiBi bias at equilibrium (fractional) positions, every kernel
+    that serves the entry point: fp32 / head_dim 64 SIMT, bf16 tensor-core, bf16 query-only."""
+    rng = np.random.default_rng(5)
+    lay = build_layout([0, 40, 130], [[1, 15, 70, 200], [17, 127, 0], [128, 300]],
+                       [[9, 9, 9, 9], [33, 33, 33], [24, 24]])
+    H, Hkv, T = 4, 2, lay.total_tokens
+    pos, _ = positions_for(lay, lambda P, L, Q: oracle.positions(P, L, Q))
+    slopes = _slopes(H) * 4.0
+    q, k, v = _randn((T, H, D), dtype, 31), _randn((T, Hkv, D), dtype, 32), _randn((T, Hkv, D), dtype, 33)
+    scale = 1 / math.sqrt(D)
+    ref_o, ref_l = oracle.prefill(f32(q), f32(k), f32(v), lay, scale, pos=pos, slopes=slopes)
+    plain_o, _ = oracle.prefill(f32(q), f32(k), f32(v), lay, scale)
+    assert rel_l2(plain_o, ref_o) > 0.05, "the bias must matter in this test"
+    dl = sp.DeviceLayout.from_host(lay)
+    qd = dev(q)
+    out = torch.full_like(qd, float("nan"))
+    lse = torch.full((H, T), float("nan"), device="cuda")
+    ws = workspace(sp.sp_prefill_workspace_bytes(dl, H, D, sp.dtype_code(qd)))
+    mode = sp.SP_ROWS_ALL if rows == "all" else sp.SP_ROWS_QUERY_ONLY
+    sp.sp_superpose_prefill_alibi(qd, dev(k), dev(v), dl, dev(pos), dev(slopes), scale, out, lse, ws, rows=mode)
+    sp.sp_check_status(ws)
+    sel = np.ones(T, bool) if rows == "all" else _query_row_mask(lay)
+    got_o, got_l = f32(out), lse.cpu().numpy()
+    assert np.isnan(got_o[~sel]).all() and not np.isnan(got_o[sel]).any()
+    assert rel_l2(got_o[sel], ref_o[sel]) <= TOL[dtype]
+    num = np.linalg.norm((got_o - ref_o)[sel].reshape(int(sel.sum()), -1), axis=1)
+    den = np.linalg.norm(ref_o[sel].reshape(int(sel.sum()), -1), axis=1) + 1e-6
+    assert (num / den).max() <= 5 * TOL[dtype]
+    np.testing.assert_allclose(got_l[:, sel], ref_l[:, sel], atol=2e-5 if dtype == "f32" else 2e-2)
+
+
+@pytest.mark.parametrize("dtype,D", [("f32", 64), ("bf16", 128)])
+def test_decode_alibi_parity(dtype, D):
+    lay = build_layout([16, 3], [[32, 1, 129, 40], [200, 17]], [[8, 8, 8, 8], [5, 5]])
+    B, H, Hkv, T, k_top, cap = 2, 4, 2, lay.total_tokens, 2, 6
+    kc, vc = _randn((T, Hkv, D), dtype, 41), _randn((T, Hkv, D), dtype, 42)
+    q = _randn((B, H, D), dtype, 43)
+    tk, tv = _randn((B, cap, Hkv, D), dtype, 44), _randn((B, cap, Hkv, D), dtype, 45)
+    kept = np.array([[2, 0], [4, -1]], np.int32)
+    tl = np.array([6, 1], np.int32)
+    cpos, nxt = positions_for(lay, lambda P, L, Q: oracle.positions(P, L, Q))
+    tpos = (nxt[:, None] + np.arange(cap)[None, :]).astype(np.float32)
+    qpos = tpos[np.arange(B), tl - 1].copy()
+    slopes = _slopes(H) * 4.0
+    scale = 1 / math.sqrt(D)
+    ref_o, ref_l = oracle.pruned_decode(f32(q), f32(kc), f32(vc), lay, kept, f32(tk), f32(tv), tl, scale,
+                                        q_pos=qpos, cache_pos=cpos, tail_pos=tpos, slopes=slopes)
+    plain_o, _ = oracle.pruned_decode(f32(q), f32(kc), f32(vc), lay, kept, f32(tk), f32(tv), tl, scale)
+    assert rel_l2(plain_o, ref_o) > 0.05
+    dl = sp.DeviceLayout.from_host(lay)
+    out = torch.full((B, H, D), float("nan"), dtype=TDT[dtype], device="cuda")
+    lse = torch.full((B, H), float("nan"), device="cuda")
+    ws = workspace(sp.sp_decode_workspace_bytes(B, H, D))
+    sp.sp_pruned_decode_alibi(dev(q), dev(kc), dev(vc), dl, dev(kept), k_top, dev(tk), dev(tv), dev(tl), cap,
+                              dev(qpos), dev(cpos), dev(tpos), dev(slopes), scale, out, lse, ws)
+    sp.sp_check_status(ws)
+    assert rel_l2(f32(out), ref_o) <= TOL[dtype]
+    np.testing.assert_allclose(lse.cpu().numpy(), ref_l, atol=2e-5 if dtype == "f32" else 2e-2)
