@@ -99,6 +99,16 @@ int sp_rope_apply(void *x, const float *pos, int64_t n_tokens, int64_t ld_token,
                   int head_dim, int rot_dim, double base, int pairing, int dtype, void *stream);
 
 /*
+ * The same rotation for two tensors that share their positions, in one launch: a step's
+ * queries xq [n_tokens, n_heads_q, head_dim] (token stride ld_q) and keys xk [n_tokens,
+ * n_heads_k, head_dim] (token stride ld_k).  Each angle is evaluated once for both.
+ * Equivalent to two sp_rope_apply calls; same argument rules, same dtype for both tensors.
+ */
+int sp_rope_apply_pair(void *xq, int64_t ld_q, int n_heads_q, void *xk, int64_t ld_k, int n_heads_k,
+                       const float *pos, int64_t n_tokens, int head_dim, int rot_dim, double base,
+                       int pairing, int dtype, void *stream);
+
+/*
  * Fork-join ("superposition") prefill attention (Section 3.2: a segment attends to
  * another iff the prompt DAG has a path to it; ForkJoin topology preamble -> documents ->
  * query copies; every call is dense causal attention on its own tokens plus the KV of

@@ -29,7 +29,7 @@ EXPORTS = (
     "sp_path_scores_workspace_bytes", "sp_path_scores", "sp_prune_topk",
     "sp_decode_workspace_bytes", "sp_pruned_decode", "sp_check_status",
     "sp_pruned_decode_static_max_bytes", "sp_pruned_decode_static",
-    "sp_superpose_prefill_alibi", "sp_pruned_decode_alibi",
+    "sp_superpose_prefill_alibi", "sp_pruned_decode_alibi", "sp_rope_apply_pair",
 )
 
 
@@ -63,6 +63,7 @@ def _load() -> ctypes.CDLL:
     lib.sp_version.restype = ctypes.c_char_p
     lib.sp_positions.argtypes = [c_int, c_int, c_int, c_int, vp, c_int, vp, ctypes.POINTER(c_d), ctypes.POINTER(c_d)]
     lib.sp_rope_apply.argtypes = [vp, vp, c_i64, c_i64, c_int, c_int, c_int, c_d, c_int, c_int, vp]
+    lib.sp_rope_apply_pair.argtypes = [vp, c_i64, c_int, vp, c_i64, c_int, vp, c_i64, c_int, c_int, c_d, c_int, c_int, vp]
     lib.sp_prefill_workspace_bytes.argtypes = [c_int] * 7
     lib.sp_prefill_workspace_bytes.restype = sz
     lib.sp_superpose_prefill.argtypes = [vp, vp, vp, lp, c_int, c_int, c_int, c_f, c_int, vp, vp, vp, sz, c_int, vp]
@@ -169,6 +170,17 @@ def sp_rope_apply(x: torch.Tensor, pos: torch.Tensor, n_heads: int, head_dim: in
     _check(lib.sp_rope_apply(x.data_ptr(), pos.data_ptr(), n, ld, n_heads, head_dim,
                              head_dim if rot_dim is None else rot_dim, base, pairing, dtype_code(x),
                              _stream(stream)))
+
+
+def sp_rope_apply_pair(xq: torch.Tensor, n_heads_q: int, xk: torch.Tensor, n_heads_k: int, pos: torch.Tensor,
+                       head_dim: int, *, n_tokens=None, ld_q=None, ld_k=None, rot_dim=None, base: float = 10000.0,
+                       pairing: int = SP_ROPE_HALF_SPLIT, stream=None):
+    """sp_rope_apply on a step's queries and keys (same positions) in one launch, in place."""
+    n = pos.numel() if n_tokens is None else n_tokens
+    _check(lib.sp_rope_apply_pair(xq.data_ptr(), n_heads_q * head_dim if ld_q is None else ld_q, n_heads_q,
+                                  xk.data_ptr(), n_heads_k * head_dim if ld_k is None else ld_k, n_heads_k,
+                                  pos.data_ptr(), n, head_dim, head_dim if rot_dim is None else rot_dim, base,
+                                  pairing, dtype_code(xq), _stream(stream)))
 
 
 def sp_prefill_workspace_bytes(lay: DeviceLayout, n_heads: int, head_dim: int, dtype: int) -> int:

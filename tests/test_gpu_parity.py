@@ -61,6 +61,27 @@ def test_rope_strided_tokens_and_empty():
     sp.sp_rope_apply(bd, dev(pos), H, D, n_tokens=0)      # no-op
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_rope_pair_equals_two_calls(dtype):
+    """Queries and keys of a step rotated in one launch: bit-identical to two single calls, also
+    with different head counts, a strided key tensor and an unaligned (scalar-path) shape."""
+    for (Hq, Hk, D, rot, n, ldk) in [(32, 8, 128, 128, 301, None), (4, 4, 64, 32, 5, 3 * 4 * 64), (3, 1, 24, 12, 9, None)]:
+        xq, xk = _randn((n, Hq, D), dtype, 70), _randn((n, (ldk or Hk * D)), dtype, 71)
+        pos = (torch.rand(n, generator=_rng(72)) * 900).float()
+        q1, k1 = dev(xq), dev(xk)
+        sp.sp_rope_apply(q1, dev(pos), Hq, D, rot_dim=rot)
+        sp.sp_rope_apply(k1, dev(pos), Hk, D, rot_dim=rot, ld_token=ldk)
+        q2, k2 = dev(xq), dev(xk)
+        sp.sp_rope_apply_pair(q2, Hq, k2, Hk, dev(pos), D, rot_dim=rot, ld_k=ldk)
+        assert torch.equal(q1, q2) and torch.equal(k1, k2)
+        ref = oracle.rope(f32(xq), pos.numpy(), rot_dim=rot)
+        tol = 4e-6 if dtype == "f32" else None
+        if tol:
+            np.testing.assert_allclose(f32(q2), ref, rtol=0, atol=tol)
+        else:
+            assert np.all(np.abs(f32(q2) - ref) <= np.abs(ref) * 2.0 ** -8 * 1.02 + 1e-6)
+
+
 # ------------------------------------------------------------------------- prefill
 def _prefill_gpu(q, k, v, lay, scale, rows=sp.SP_ROWS_ALL, poison=True):
     dl = sp.DeviceLayout.from_host(lay)
