@@ -40,7 +40,7 @@ PREFILL_LAUNCHES = 2           # kernels sp_superpose_prefill launches per call 
 # the ncu captures summarised under profiles/ (absent = not captured for the current kernel).
 NCU_TRAFFIC_BYTES = {
     # scaled by tokens / prompts from the 20-prompt captures (traffic grows in proportion)
-    ("prefill", "cfg2_batched_serving"): 9.016e9,
+    ("prefill", "cfg2_batched_serving"): 9.077e9,
     ("decode", "cfg2_batched_serving"): 4.407e8,
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}

@@ -105,7 +105,7 @@ __device__ __forceinline__ void rotate_tokens(T *__restrict__ x, const float2 (*
 // One launch may rotate two tensors that share their positions (a step's Q and K): x1 == NULL
 // rotates x alone.  VEC / VEC1: whether the 16-byte path applies to x / x1.
 template <typename T, bool VEC, bool VEC1>
-__global__ void __launch_bounds__(kRopeThreads)
+__global__ void __launch_bounds__(kRopeThreads, 8)   // 32 registers: full occupancy for the streaming pass
 rope_kernel(T *__restrict__ x, T *__restrict__ x1, const float *__restrict__ pos, int64_t n_tokens, int64_t ld_token,
             int64_t ld_token1, int n_heads, int n_heads1, int head_dim, int rot_dim, int pairing,
             const __grid_constant__ RopeFreq fr)
