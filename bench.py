@@ -41,7 +41,7 @@ PREFILL_LAUNCHES = 2           # kernels sp_superpose_prefill launches per call 
 NCU_TRAFFIC_BYTES = {
     # scaled by tokens / prompts from the 20-prompt captures (traffic grows in proportion)
     ("prefill", "cfg2_batched_serving"): 9.077e9,
-    ("decode", "cfg2_batched_serving"): 4.407e8,
+    ("decode", "cfg2_batched_serving"): 4.389e8,
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
