@@ -262,7 +262,7 @@ def test_prefill_is_deterministic():
         np.testing.assert_array_equal(la, lb)
 
 
-@pytest.mark.parametrize("case", ["mixed", "tiny_items", "preamble_only"])
+@pytest.mark.parametrize("case", ["mixed", "tiny_items", "preamble_only", "merged_documents"])
 def test_prefill_random_ragged_layouts(case):
     """Random segment lengths (empty documents and preambles included), grouped-query heads,
     items of every size next to each other in the persistent blocks' work lists."""
@@ -275,6 +275,12 @@ def test_prefill_random_ragged_layouts(case):
         lay = build_layout([0] * 4, [list(rng.integers(0, 30, 200)) for _ in range(4)],
                            [list(rng.integers(1, 8, 200)) for _ in range(4)])
         H, Hkv = 4, 4
+    elif case == "merged_documents":
+        # superposition factor > 1 (Appendix ablation): several documents share a path, so paths
+        # run to many query tiles and long causal key ranges
+        lay = build_layout([48, 0], [list(rng.integers(500, 1000, 5)), list(rng.integers(300, 700, 4))],
+                           [[32] * 5, [24] * 4])
+        H, Hkv = 4, 2
     else:
         lay = build_layout([700, 1, 129], [[], [], []], [[], [], []])
         H, Hkv = 4, 1
