@@ -5,9 +5,9 @@
 // (all visible) followed by the segment's own rows up to the diagonal; key tiles that the
 // fork-join mask excludes are never loaded or multiplied.  Per key tile of up to 64 keys:
 //   S = Q K^T     tcgen05.mma, A and B from TMA-staged 128B-swizzled shared memory, fp32 in TMEM
-//   P = softmax   4 warps, one thread per query row (tcgen05.ld, the tile's scores stay in
-//                 registers), online max / sum with lazy rescaling, P rounded to bf16 and written
-//                 over S in TMEM (tcgen05.st)
+//   P = softmax   4 warps, one thread per query row; two rolled passes over the tile in chunks of
+//                 16 keys (tcgen05.ld): row maximum, then exp2 / sum with lazy rescaling, P rounded
+//                 to bf16 and written over S in TMEM (tcgen05.st)
 //   O += P V      tcgen05.mma with A = P from TMEM, B = V from shared memory (MN-major)
 // Roles (warpgroups of 4 warps, registers rebalanced with setmaxnreg): warps 0-3 softmax,
 // warps 4-7 epilogue (O / l -> bf16 -> global, LSE) off the softmax warps' critical path,
@@ -35,9 +35,14 @@ constexpr int kTcThreads = 12 * 32;   // warps 0-3 softmax, 4-7 epilogue, 8 prod
 constexpr int kQBytes = kBM * kHD * 2;     // 32 KB
 constexpr int kKVBytes = kBN * kHD * 2;    // 16 KB per stage
 constexpr int kTmemCols = 256;        // S/P double buffer: [0,64) [64,128)   O: [128,256)
+constexpr int kCh = 16;               // keys per softmax chunk
 constexpr float kLog2eT = 1.4426950408889634f;
 constexpr float kLn2T = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.f;   // log2 units: rescale O only when the max grows by > 2^8
+
+static_assert(kCh == 16, "the chunk loads and stores below are the 16-column forms");
+__device__ __forceinline__ void tmem_ldc(uint32_t a, uint32_t (&r)[16]) { tmem_ld16(a, r); }
+__device__ __forceinline__ void tmem_stc(uint32_t a, const uint32_t (&r)[8]) { tmem_st8(a, r); }
 
 __device__ __forceinline__ float ex2(float x)
 {
@@ -284,7 +289,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
         __syncwarp();
     } else if (warp < 4) {
         // ------------------------------------------------------------------ softmax
-        // One thread per query row; a tile's 64 scores stay in registers (one TMEM read).
+        // One thread per query row.
         reg_alloc<120>();
         const int row = warp * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
@@ -309,8 +314,6 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             // A warp whose 32 rows lie past the tile's last valid row does no arithmetic at all:
             // its rows of P and O are never stored (it still takes part in every barrier).
             const bool live_w = warp * 32 < t.n_rows;
-            const bool use0 = live_w && lim31 > 0;               // uniform: keys [0,32) seen by some row
-            const bool use1 = live_w && lim31 > 32;              // uniform: keys [32,64) seen by some row
             if (first) {
                 m_ref = -INFINITY; l = 0.f;
                 if (ALIBI) {
@@ -321,44 +324,32 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
             tc_fence_after();
 
-            uint32_t r0[32], r1[32];
-            if (use0) tmem_ld32(s_addr, r0);
-            if (use1) tmem_ld32(s_addr + 32, r1);
-            tmem_ld_wait();
-            // keys past the row's limit (causal diagonal, ragged tail) -> -inf; skipped when the
-            // whole warp sees everything it loaded
+            // The tile is walked twice in chunks of 16 keys (rolled loops, scores re-read from tensor
+            // memory): the code of this role stays small, which matters more than the second read.
+            // n_ch chunks are read by the MMA; `see` of them hold keys some row of this warp may see.
+            const int n_ch = (n_mma + kCh - 1) / kCh;
+            const int see = live_w ? min(n_ch, (max(lim31, 0) + kCh - 1) / kCh) : 0;
             float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            if (ALIBI) {                // score * scale - slope * |distance|, every thread reads the same key positions
-                if (use0) {
+#pragma unroll 1
+            for (int ch = 0; ch < see; ++ch) {          // pass 1: the row's maximum over the tile
+                uint32_t r[kCh];
+                tmem_ldc(s_addr + ch * kCh, r);
+                tmem_ld_wait();
+                if (ALIBI) {            // score * scale - slope * |distance|, every thread reads the same key positions
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float pk = i < kt.n_valid ? __ldg(p.pos + kt.row0 + i) : 0.f;
-                        r0[i] = __float_as_uint(fmaf(__uint_as_float(r0[i]), sc, -slope_l2 * fabsf(pq - pk)));
+                    for (int i = 0; i < kCh; ++i) {
+                        const float pk = ch * kCh + i < kt.n_valid ? __ldg(p.pos + kt.row0 + ch * kCh + i) : 0.f;
+                        r[i] = __float_as_uint(fmaf(__uint_as_float(r[i]), sc, -slope_l2 * fabsf(pq - pk)));
                     }
                 }
-                if (use1) {
+                // keys past the row's limit (causal diagonal, ragged tail) -> -inf; skipped when the
+                // whole warp sees the whole chunk
+                if (ch * kCh + 16 > lim0) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float pk = 32 + i < kt.n_valid ? __ldg(p.pos + kt.row0 + 32 + i) : 0.f;
-                        r1[i] = __float_as_uint(fmaf(__uint_as_float(r1[i]), sc, -slope_l2 * fabsf(pq - pk)));
-                    }
-                }
-            }
-            if (use0) {
-                if (lim0 < 32) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) r0[i] = (i < lim) ? r0[i] : 0xff800000u;
+                    for (int i = 0; i < kCh; ++i) r[i] = (ch * kCh + i < lim) ? r[i] : 0xff800000u;
                 }
 #pragma unroll
-                for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(r0[i]));
-            }
-            if (use1) {
-                if (lim0 < 64) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) r1[i] = (32 + i < lim) ? r1[i] : 0xff800000u;
-                }
-#pragma unroll
-                for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(r1[i]));
+                for (int i = 0; i < kCh; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(r[i]));
             }
             const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc_exp;
             float alpha = 1.f;
@@ -389,47 +380,37 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 // masked scores are -inf, so exp2 gives exactly 0 for them
                 const float nm = -m_ref;
                 float rs[4] = {0.f, 0.f, 0.f, 0.f};
-                if (use0) {
+#pragma unroll 1
+                for (int ch = 0; ch < n_ch; ++ch) {     // pass 2: P = exp2(score - reference) as bf16, written over S
+                    uint32_t pk[kCh / 2];
+                    if (ch < see) {
+                        uint32_t r[kCh];
+                        tmem_ldc(s_addr + ch * kCh, r);
+                        tmem_ld_wait();
+                        if (ALIBI) {
 #pragma unroll
-                    for (int q8 = 0; q8 < 2; ++q8) {              // 16 keys -> 8 packed pairs per store
-                        uint32_t pk[8];
+                            for (int i = 0; i < kCh; ++i) {
+                                const float pkey = ch * kCh + i < kt.n_valid ? __ldg(p.pos + kt.row0 + ch * kCh + i) : 0.f;
+                                r[i] = __float_as_uint(fmaf(__uint_as_float(r[i]), sc, -slope_l2 * fabsf(pq - pkey)));
+                            }
+                        }
+                        if (ch * kCh + 16 > lim0) {
 #pragma unroll
-                        for (int i = 0; i < 16; i += 2) {
-                            const float p0 = ex2(fmaf(__uint_as_float(r0[q8 * 16 + i]), sc_exp, nm));
-                            const float p1 = ex2(fmaf(__uint_as_float(r0[q8 * 16 + i + 1]), sc_exp, nm));
+                            for (int i = 0; i < kCh; ++i) r[i] = (ch * kCh + i < lim) ? r[i] : 0xff800000u;
+                        }
+#pragma unroll
+                        for (int i = 0; i < kCh; i += 2) {
+                            const float p0 = ex2(fmaf(__uint_as_float(r[i]), sc_exp, nm));
+                            const float p1 = ex2(fmaf(__uint_as_float(r[i + 1]), sc_exp, nm));
                             rs[(i >> 1) & 3] += p0 + p1;
                             pk[i >> 1] = pack_bf16x2(p0, p1);
                         }
-                        tmem_st8(s_addr + q8 * 8, pk);
+                    } else {                            // keys no row of this warp sees
+#pragma unroll
+                        for (int i = 0; i < kCh / 2; ++i) pk[i] = 0u;
                     }
-                } else {
-                    uint32_t z[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) z[i] = 0u;
-                    tmem_st8(s_addr, z);
-                    tmem_st8(s_addr + 8, z);
-                }
-                if (n_mma > 32) {
-                    if (use1) {
-#pragma unroll
-                        for (int q8 = 0; q8 < 2; ++q8) {
-                            uint32_t pk[8];
-#pragma unroll
-                            for (int i = 0; i < 16; i += 2) {
-                                const float p0 = ex2(fmaf(__uint_as_float(r1[q8 * 16 + i]), sc_exp, nm));
-                                const float p1 = ex2(fmaf(__uint_as_float(r1[q8 * 16 + i + 1]), sc_exp, nm));
-                                rs[(i >> 1) & 3] += p0 + p1;
-                                pk[i >> 1] = pack_bf16x2(p0, p1);
-                            }
-                            tmem_st8(s_addr + 16 + q8 * 8, pk);
-                        }
-                    } else {
-                        uint32_t z[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) z[i] = 0u;
-                        tmem_st8(s_addr + 16, z);
-                        tmem_st8(s_addr + 24, z);
-                    }
+                    // P chunk ch (8 columns of bf16 pairs) lands on score columns already consumed
+                    tmem_stc(s_addr + ch * (kCh / 2), pk);
                 }
                 l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
             }
