@@ -30,7 +30,7 @@ using namespace ptx;
 constexpr int kBM = 128;              // query rows per tile
 constexpr int kBN = 64;               // keys per tile
 constexpr int kHD = 128;              // head_dim
-constexpr int kTmaWarp = 8, kMmaWarp = 9;
+constexpr int kTmaWarp = 8, kMmaWarp = 9, kCleanWarp = 10;
 constexpr int kTcThreads = 12 * 32;   // warps 0-3 softmax, 4-7 epilogue, 8 producer, 9 MMA issuer, 10-11 idle (warpgroup padding)
 constexpr int kQBytes = kBM * kHD * 2;     // 32 KB
 constexpr int kKVBytes = kBN * kHD * 2;    // 16 KB per stage
@@ -141,9 +141,11 @@ struct Cursor {
 // the current item before the warp on the diagonal has published its rows.
 // O_FREE: the epilogue warps have read the item's O out of tensor memory, so the next item's
 // first O = P V may overwrite it.
+// V_CLEAN[st]: on a tile whose key count is not a multiple of 16, the rows of the V stage between the
+// last key and the end of the last 16-key MMA step have been zeroed (see the cleaner role).
 enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_V_FULL = BAR_K_FULL + 2, BAR_S_FULL = BAR_V_FULL + 2,
        BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2, BAR_L_READY = BAR_O_DONE + 2,
-       BAR_X_FREE = BAR_L_READY + 2, BAR_O_FREE = BAR_X_FREE + 2, BAR_DRAIN, BAR_COUNT };
+       BAR_X_FREE = BAR_L_READY + 2, BAR_O_FREE = BAR_X_FREE + 2, BAR_V_CLEAN, BAR_DRAIN = BAR_V_CLEAN + 2, BAR_COUNT };
 
 template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
@@ -181,7 +183,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
     bool ok = true;
 
     if (warp >= 8) {
-        reg_dealloc<40>();              // warps 8-11: producer, MMA issuer and two idle warps
+        reg_dealloc<56>();              // warps 8-11: producer, MMA issuer and two idle warps
         if (warp == kTmaWarp) {
             // -------------------------------------------------------------- TMA producer
             if (lane == 0) {
@@ -229,6 +231,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 const uint32_t k_lo = ((smem_u32(sK) & 0x3ffffu) >> 4) | (1u << 16);
                 const uint32_t v_lo = (smem_u32(sV) & 0x3ffffu) >> 4;     // leading-dimension offset (half stride) added per tile
                 const uint32_t id_o = idesc_bf16(kBM, kHD, 0, 1);
+                uint32_t n_ragged[2] = {0, 0};      // ragged tiles seen per V stage (phase of V_CLEAN)
                 Cursor cs, cp;                      // cs: next S = Q K^T to issue; cp: next O += P V to issue
                 cs.init(p.tiles, n_items, p.n_heads);
                 cp.init(p.tiles, n_items, p.n_heads);
@@ -266,6 +269,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     const int n_k = (pv_valid + 15) >> 4;                 // 16-key steps
                     if (!(ok = mbar_wait(&bars[BAR_P_FULL + st], ph))) break;
                     if (!(ok = mbar_wait(&bars[BAR_V_FULL + st], ph))) break;
+                    if ((pv_valid & 15) && !(ok = mbar_wait(&bars[BAR_V_CLEAN + st], n_ragged[st]++ & 1))) break;
                     // the first O = P V of an item overwrites O: the previous item's must have been read out
                     if (cp.j == 0 && cp.item_no > 0 && !(ok = mbar_wait(&bars[BAR_O_FREE], (cp.item_no - 1) & 1))) break;
                     tc_fence_after();
@@ -285,12 +289,43 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     mbar_wait(&bars[BAR_DRAIN], 0);
                 }
             }
+        } else if (warp == kCleanWarp) {
+            // -------------------------------------------------------------- V cleaner
+            // O += P V contracts over the keys rounded up to 16.  The rows of the V stage past the
+            // tile's last key hold whatever follows in the packed tensor (another path's rows);
+            // their P is exactly zero, but 0 x Inf or 0 x NaN would still reach O.  This warp
+            // zeroes those rows before the issuer may use the stage, so a path's output depends on
+            // nothing outside its own keys (Section 3.2: paths do not see each other).
+            uint32_t n_ragged[2] = {0, 0};
+            Cursor c;
+#pragma unroll 1
+            for (c.init(p.tiles, n_items, p.n_heads); c.valid && ok; c.next()) {
+                const int n_valid = c.kv().n_valid;
+                const int st = c.g & 1;
+                // every tile's phase is waited for (not only the ragged ones), so that this warp can
+                // never be a whole barrier phase ahead of the loads
+                if (!(ok = mbar_wait_warp(&bars[BAR_V_FULL + st], (c.g >> 1) & 1))) break;
+                if ((n_valid & 15) == 0) continue;
+                const int n_mma = (n_valid + 15) & ~15;
+                const int half_bytes = (32 << kv_box_sel(n_valid)) * 128;      // one 64-column half of the box
+                unsigned char *vs = sV + st * kKVBytes;
+                // (rows n_valid .. n_mma-1) x 2 halves x 8 pieces of 16 bytes; the 128-byte swizzle only
+                // permutes the pieces inside a row
+                for (int i = lane; i < (n_mma - n_valid) * 16; i += 32) {
+                    const int r = n_valid + (i >> 4), half = (i >> 3) & 1, piece = i & 7;
+                    *reinterpret_cast<uint4 *>(vs + half * half_bytes + r * 128 + piece * 16) = make_uint4(0u, 0u, 0u, 0u);
+                }
+                fence_proxy_async();                 // generic-proxy stores -> visible to the MMA's reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars[BAR_V_CLEAN + st]);
+                ++n_ragged[st];
+            }
         }
         __syncwarp();
     } else if (warp < 4) {
         // ------------------------------------------------------------------ softmax
         // One thread per query row.
-        reg_alloc<120>();
+        reg_alloc<104>();
         const int row = warp * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
         const float sc = p.scale_log2e;
@@ -321,7 +356,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     slope_l2 = p.slopes[c.h] * kLog2eT;
                 }
             }
-            if (!(ok = mbar_wait(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
+            if (!(ok = mbar_wait_warp(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
             tc_fence_after();
 
             // The tile is walked twice in chunks of 16 keys (rolled loops, scores re-read from tensor
@@ -363,7 +398,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             }
             if (__any_sync(0xffffffffu, grow)) {     // rare: bring O and l to the new reference
                 // needs the previous tile's O += P V complete
-                if (!(ok = mbar_wait(&bars[BAR_O_DONE + ((c.g - 1) & 1)], ((c.g - 1) >> 1) & 1))) break;
+                if (!(ok = mbar_wait_warp(&bars[BAR_O_DONE + ((c.g - 1) & 1)], ((c.g - 1) >> 1) & 1))) break;
                 tc_fence_after();
                 l *= alpha;
 #pragma unroll 1
@@ -421,7 +456,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             if (c.last_of_item()) {                 // hand the item's row statistics to the epilogue warps
                 const uint32_t xp = c.item_no & 1;
                 // the slot was last used two items ago: the epilogue must have read it
-                if (c.item_no >= 2 && !(ok = mbar_wait(&bars[BAR_X_FREE + xp], ((c.item_no >> 1) - 1) & 1))) break;
+                if (c.item_no >= 2 && !(ok = mbar_wait_warp(&bars[BAR_X_FREE + xp], ((c.item_no >> 1) - 1) & 1))) break;
                 x_l[xp][row] = l;
                 x_m[xp][row] = m_ref;
                 mbar_arrive(&bars[BAR_L_READY + xp]);
@@ -445,10 +480,10 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             g_end += (t.pre_len + kBN - 1) / kBN + (t.q_off + t.n_rows + kBN - 1) / kBN;
             const uint32_t g_last = g_end - 1;
             const int xp = item_no & 1;
-            if (!(ok = mbar_wait(&bars[BAR_L_READY + xp], (item_no >> 1) & 1))) break;
+            if (!(ok = mbar_wait_warp(&bars[BAR_L_READY + xp], (item_no >> 1) & 1))) break;
             const float l_row = x_l[xp][row], m_row = x_m[xp][row];
             mbar_arrive(&bars[BAR_X_FREE + xp]);
-            if (!(ok = mbar_wait(&bars[BAR_O_DONE + (g_last & 1)], (g_last >> 1) & 1))) break;   // last O += P V
+            if (!(ok = mbar_wait_warp(&bars[BAR_O_DONE + (g_last & 1)], (g_last >> 1) & 1))) break;   // last O += P V
             tc_fence_after();
             const float inv = 1.f / l_row;
             unsigned char *dst = reinterpret_cast<unsigned char *>(p.out) + ((int64_t)t.q_row * p.n_heads + h) * (kHD * 2);

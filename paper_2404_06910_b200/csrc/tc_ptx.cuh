@@ -49,14 +49,34 @@ __device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity)
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: false when the limit ran out (the caller records a timeout and unwinds).
-constexpr uint32_t kWaitLimit = 1u << 21;   // about two seconds at the hint above
+// Bounded wait: false when the time limit ran out (the caller records a timeout and unwinds).
+constexpr uint64_t kWaitLimitNs = 2000000000ull;      // two seconds of the global nanosecond timer
+__device__ __forceinline__ uint64_t global_timer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
 {
-    for (uint32_t i = 0; i < kWaitLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+#pragma unroll 1                            // left to itself the compiler unrolls this loop at every call site
+    while (!mbar_try_wait(bar, parity))
+        if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+    return true;
 }
+
+// The same wait for whole warps that go on to warp-aligned tcgen05 instructions: the outcome
+// is made uniform, so a limit that runs out for some lanes only cannot split the warp.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity)
+{
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity));
+}
+
+// Orders this thread's ordinary shared-memory stores before later reads by the asynchronous
+// proxy (TMA, tcgen05.mma).
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---- TMA -------------------------------------------------------------------------------
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap *m)
