@@ -199,6 +199,7 @@ class HotPath:
         # per decode step rope (q and the new key in one launch) + decode
         self.launches = 2 + PREFILL_LAUNCHES + 2 + 1 + self.steps_dec * 2
         self.decode_graph = None
+        self.fused_rope = (H // Hkv) in (1, 2, 4)
         self.kv_sets = [(self.k, self.v)]
 
     def decode_bytes(self):
@@ -260,10 +261,16 @@ class HotPath:
         H, Hkv, D, B = self.H, self.Hkv, self.D, self.B
         ld = self.steps_dec * Hkv * D
         for t in range(self.steps_dec):
+            kc, vc = self.kv_sets[t % len(self.kv_sets)]
+            if with_rope and self.fused_rope:
+                # one launch per token: the new query and key rows are rotated inside the decode kernel
+                sp.sp_pruned_decode_rope(self.dq[t], kc, vc, self.dl, self.kept, cfg.top_k, self.tk, self.tv,
+                                         self.tail_len[t], self.steps_dec, self.tpos[t], self.scale, self.dec_out[t],
+                                         None, base=cfg.rope_base)
+                continue
             if with_rope:
                 sp.sp_rope_apply_pair(self.dq[t], H, self.tk[:, t], Hkv, self.tpos[t], D, n_tokens=B, ld_k=ld,
                                       base=cfg.rope_base)
-            kc, vc = self.kv_sets[t % len(self.kv_sets)]
             sp.sp_pruned_decode(self.dq[t], kc, vc, self.dl, self.kept, cfg.top_k, self.tk, self.tv,
                                 self.tail_len[t], self.steps_dec, self.scale, self.dec_out[t], None, self.ws_dec)
 

@@ -178,7 +178,12 @@ int sp_prune_topk(const float *scores, const int32_t *prompt_path_off, int n_pro
  * A prompt with no key at all gets out = 0 and lse = -inf.
  * max_keys: host upper bound on any prompt's key count (sizes the KV split);
  * pass 0 to use max_pre_len + k * max_path_len + tail_cap.
- * ws: at least sp_decode_workspace_bytes() bytes, 256-byte aligned.
+ * ws: at least sp_decode_workspace_bytes() bytes, 256-byte aligned.  The key sequence of a
+ * (prompt, KV head) is split over the blocks of one thread-block cluster, which merge their
+ * partial results through distributed shared memory in split order (results do not depend on
+ * scheduling); the workspace is therefore not written, and its status word is not touched
+ * (this call has no bounded waits).  Query heads that share a KV head (n_kv_heads < n_heads) are
+ * served by one block per KV head, in groups of 4, 2 or 1, so K and V rows are read once per group.
  */
 size_t sp_decode_workspace_bytes(int n_prompts, int n_heads, int head_dim);
 int sp_pruned_decode(const void *q, const void *k_cache, const void *v_cache,
@@ -212,6 +217,27 @@ int sp_pruned_decode_alibi(const void *q, const void *k_cache, const void *v_cac
                            const float *tail_pos, const float *slopes, int n_heads, int n_kv_heads,
                            int head_dim, float scale, void *out, float *lse, void *ws, size_t ws_bytes,
                            int dtype, void *stream);
+
+/*
+ * Decode step with the rotary embedding folded in (Section 3.2.2 footnote: the sinusoid is
+ * evaluated at the token's real-valued position).  Computes what
+ *   sp_rope_apply_pair(q, newest tail key, positions q_pos)  followed by  sp_pruned_decode
+ * computes, in one launch: q [B, n_heads, D] and the newest tail key row
+ * tail_k[b][tail_len[b] - 1] arrive unrotated; both are rotated at position q_pos[b] (fp32 [B],
+ * device; angles formed in fp64, results rounded to the storage type as the stand-alone
+ * rotation does), and the rotated key row is written back in place, so later steps find it
+ * rotated like every older row.  q itself is not modified.  A prompt with tail_len[b] == 0 has
+ * no new key.  rope_base > 0; pairing as in sp_rope_apply; the rotation spans the whole head
+ * (rot_dim == head_dim).  n_heads / n_kv_heads must be 1, 2 or 4 (one block has to own the new
+ * key row); other ratios return SP_ERR_UNSUPPORTED: rotate separately and call
+ * sp_pruned_decode.  No workspace; all other arguments as for sp_pruned_decode.
+ */
+int sp_pruned_decode_rope(const void *q, const void *k_cache, const void *v_cache,
+                          const sp_layout *lay, const int32_t *kept_idx, int k, void *tail_k,
+                          const void *tail_v, const int32_t *tail_len, int tail_cap, int64_t max_keys,
+                          const float *q_pos, double rope_base, int pairing, int n_heads,
+                          int n_kv_heads, int head_dim, float scale, void *out, float *lse, int dtype,
+                          void *stream);
 
 /*
  * Decode attention without a caller workspace.  (The paper has no counterpart: this entry

@@ -29,7 +29,7 @@ EXPORTS = (
     "sp_path_scores_workspace_bytes", "sp_path_scores", "sp_prune_topk",
     "sp_decode_workspace_bytes", "sp_pruned_decode", "sp_check_status",
     "sp_pruned_decode_static_max_bytes", "sp_pruned_decode_static",
-    "sp_superpose_prefill_alibi", "sp_pruned_decode_alibi", "sp_rope_apply_pair",
+    "sp_superpose_prefill_alibi", "sp_pruned_decode_alibi", "sp_rope_apply_pair", "sp_pruned_decode_rope",
 )
 
 
@@ -83,6 +83,8 @@ def _load() -> ctypes.CDLL:
                                                c_int, vp]
     lib.sp_pruned_decode_alibi.argtypes = [vp, vp, vp, lp, vp, c_int, vp, vp, vp, c_int, c_i64, vp, vp, vp, vp, c_int,
                                            c_int, c_int, c_f, vp, vp, vp, sz, c_int, vp]
+    lib.sp_pruned_decode_rope.argtypes = [vp, vp, vp, lp, vp, c_int, vp, vp, vp, c_int, c_i64, vp, c_d, c_int, c_int,
+                                          c_int, c_int, c_f, vp, vp, c_int, vp]
     for name in EXPORTS:
         getattr(lib, name)          # raises AttributeError if a declared symbol is not exported
     return lib
@@ -247,6 +249,19 @@ def sp_pruned_decode_alibi(q, k_cache, v_cache, lay: DeviceLayout, kept_idx, k: 
                                       _ptr(tail_k), _ptr(tail_v), _ptr(tail_len), tail_cap, max_keys, _ptr(q_pos),
                                       _ptr(cache_pos), _ptr(tail_pos), _ptr(slopes), H, Hkv, D, scale, _ptr(out),
                                       _ptr(lse), _ptr(ws), _nbytes(ws), dtype_code(q), _stream(stream)))
+
+
+def sp_pruned_decode_rope(q, k_cache, v_cache, lay: DeviceLayout, kept_idx, k: int, tail_k, tail_v, tail_len,
+                          tail_cap: int, q_pos, scale: float, out, lse=None, base: float = 10000.0,
+                          pairing: int = SP_ROPE_HALF_SPLIT, max_keys: int = 0, stream=None):
+    """One decode step with the rotary embedding folded in: q and the newest tail key row arrive
+    unrotated and are rotated at q_pos (fp32 [B]); the key row is written back rotated."""
+    B, H, D = q.shape
+    Hkv = k_cache.shape[1]
+    _check(lib.sp_pruned_decode_rope(_ptr(q), _ptr(k_cache), _ptr(v_cache), ctypes.byref(lay.c), _ptr(kept_idx), k,
+                                     _ptr(tail_k), _ptr(tail_v), _ptr(tail_len), tail_cap, max_keys, _ptr(q_pos),
+                                     base, pairing, H, Hkv, D, scale, _ptr(out), _ptr(lse), dtype_code(q),
+                                     _stream(stream)))
 
 
 def sp_pruned_decode_static_max_bytes() -> int:

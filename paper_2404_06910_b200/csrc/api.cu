@@ -21,6 +21,22 @@ int fail(int code, const char *fmt, ...)
     return code;
 }
 
+// Multiprocessor count of the current device, queried once per device; grids and split counts
+// are sized from it.  Without a usable device (host-only callers of the workspace sizers) the
+// count of the part this library is written for is assumed.
+int num_sms()
+{
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return 148; }
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) { cudaGetLastError(); n = 148; }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 int check_layout(const sp_layout *lay)
 {
     SP_REQUIRE(lay != nullptr, SP_ERR_INVALID_ARG, "layout is NULL");

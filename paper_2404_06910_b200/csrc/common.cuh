@@ -41,7 +41,7 @@ int check_layout(const sp_layout *lay);     // host-visible fields only (api.cu)
 // Device status word codes (first 4 bytes of a workspace).
 enum : uint32_t { STATUS_OK = 0, STATUS_TIMEOUT = 1 };
 
-constexpr int kNumSMs = 148;
+int num_sms();                              // multiprocessors of the current device (api.cu)
 
 // ---- device helpers ----------------------------------------------------------------
 #ifdef __CUDACC__

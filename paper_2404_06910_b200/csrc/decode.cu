@@ -7,6 +7,8 @@
 // still fill the machine; each block keeps an online softmax per key group, writes one
 // partial (max, sum, unnormalised output), and the last block to finish a (prompt, head)
 // merges the partials in split order, so results do not depend on scheduling.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace sp {
@@ -47,7 +49,7 @@ static size_t decode_counter_bytes(int n_prompts, int n_heads)
 static int decode_split_cap(int n_prompts, int n_heads)
 {
     const int64_t bh = std::max<int64_t>(1, (int64_t)n_prompts * n_heads);
-    const int64_t want = (8LL * kNumSMs) / bh;      // 8 blocks per SM: all blocks of a launch are resident at once
+    const int64_t want = (8LL * num_sms()) / bh;      // 8 blocks per SM: all blocks of a launch are resident at once
     return (int)std::min<int64_t>(kDecMaxSplits, std::max<int64_t>(1, want));
 }
 
@@ -278,6 +280,366 @@ static int launch_decode(const DecodeArgs &a, int n_prompts, cudaStream_t st)
     return a.slopes ? launch_decode_v<T, D, true>(a, n_prompts, st) : launch_decode_v<T, D, false>(a, n_prompts, st);
 }
 
+
+// ---------------------------------------------------------------------------------------
+// Cluster variant (the one sp_pruned_decode runs): the blocks that split one (prompt, KV head)
+// form a thread-block cluster and merge their partial results through distributed shared
+// memory, in split order.  No global scratch, no counters to clear, no atomics.  A block owns
+// a KV head and GRP of its query heads, so grouped heads read every K and V row once.
+// ROPE: the query rows and the newest tail key arrive unrotated and are rotated here, at the
+// new token's real-valued position (Section 3.2.2), which saves the separate launch a decode
+// step otherwise needs; the rotated key is written back to the tail for the later steps.
+// ---------------------------------------------------------------------------------------
+struct DecodeRope {
+    double inv_freq[64];      // base^(-2m/D), m < D/2 <= 64
+};
+
+template <typename T, int D, int GRP, bool ALIBI, bool ROPE>
+__global__ void __launch_bounds__(kDecThreads, GRP == 1 ? 8 : (GRP == 2 ? 5 : 3))
+decode_cluster_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ DecodeRope rope, int rope_pairing)
+{
+    namespace cg = cooperative_groups;
+    constexpr int N = Vec<T>::N;            // elements per 16-byte load
+    constexpr int LPK = D / N;              // lanes that share one key row
+    constexpr int G = kDecThreads / LPK;    // key groups per block
+    constexpr int PS = D + 2;               // one partial: D outputs, max, sum
+    static_assert(LPK <= 32 && (32 % LPK) == 0, "a key row must fit in one warp");
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int n_seg = a.k + 2;
+    int *seg_lo = reinterpret_cast<int *>(smem_raw);                        // [n_seg+1]
+    const T **seg_k = reinterpret_cast<const T **>(smem_raw + round_up((n_seg + 1) * sizeof(int), 16));
+    const T **seg_v = seg_k + n_seg;
+    const float **seg_pos = reinterpret_cast<const float **>(seg_v + n_seg);       // [n_seg], ALiBi only
+    float *red = reinterpret_cast<float *>(seg_pos + n_seg);                // [G][GRP][PS]
+    float *part = red + G * GRP * PS;                                       // [GRP][PS], read by the cluster's first block
+    float2 *cs = reinterpret_cast<float2 *>(part + GRP * PS);               // [D/2] (cos, sin), ROPE only
+
+    const int split = blockIdx.x, b = blockIdx.z;
+    const int group = a.n_heads / a.n_kv_heads;                 // query heads per KV head
+    const int per_kv = group / GRP;                             // blocks (in y) per KV head
+    const int hk = blockIdx.y / per_kv;
+    const int h0 = hk * group + (blockIdx.y - hk * per_kv) * GRP;   // first query head of this block
+    const int64_t row_elems = (int64_t)a.n_kv_heads * D;
+
+    // segments: 0 = preamble, 1..k = kept paths, k+1 = tail; lengths land in seg_lo[s+1]
+    for (int sgm = threadIdx.x; sgm < n_seg; sgm += kDecThreads) {
+        const T *kc = static_cast<const T *>(a.k_cache) + (int64_t)hk * D;
+        const T *vc = static_cast<const T *>(a.v_cache) + (int64_t)hk * D;
+        int len = 0;
+        int64_t row = 0;
+        if (sgm == 0) {
+            row = a.pre_start[b]; len = a.pre_len[b];
+        } else if (sgm <= a.k) {
+            const int i = a.kept_idx[(int64_t)b * a.k + sgm - 1];
+            if (i >= a.ppo[b] && i < a.ppo[b + 1]) { row = a.path_start[i]; len = a.doc_len[i] + a.qry_len[i]; }
+        } else {
+            len = (a.tail_cap > 0 && a.tail_len) ? min(max(a.tail_len[b], 0), a.tail_cap) : 0;
+            if (len) {
+                kc = static_cast<const T *>(a.tail_k) + (int64_t)hk * D;
+                vc = static_cast<const T *>(a.tail_v) + (int64_t)hk * D;
+                row = (int64_t)b * a.tail_cap;
+            }
+        }
+        seg_k[sgm] = kc + row * row_elems;
+        seg_v[sgm] = vc + row * row_elems;
+        if (ALIBI) seg_pos[sgm] = (sgm == a.k + 1 && len ? a.tail_pos : a.cache_pos) + row;
+        seg_lo[sgm + 1] = len;
+    }
+    if (ROPE && threadIdx.x < D / 2) {
+        // The angle is formed in fp64 at the real-valued position and brought into [-pi, pi] there
+        // (two fused steps with a split 2 pi); the small remainder goes through the fp32 sine and
+        // cosine, whose error is then far below one rounding of the rotated values.
+        const double ang = (double)a.q_pos[b] * rope.inv_freq[threadIdx.x];
+        const double turns = rint(ang * 0.15915494309189535);
+        const double r = fma(-turns, 2.4492935982947064e-16, fma(-turns, 6.283185307179586, ang));
+        float sn, cn;
+        sincosf((float)r, &sn, &cn);
+        cs[threadIdx.x] = make_float2(cn, sn);
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {                 // prefix sum of the lengths, 32 segments per round
+        int carry = 0;
+        if (threadIdx.x == 0) seg_lo[0] = 0;
+        for (int base = 0; base < n_seg; base += 32) {
+            const int sgm = base + (int)threadIdx.x;
+            int v = sgm < n_seg ? seg_lo[sgm + 1] : 0;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, v, o);
+                if ((int)threadIdx.x >= o) v += up;
+            }
+            if (sgm < n_seg) seg_lo[sgm + 1] = carry + v;
+            carry += __shfl_sync(0xffffffffu, v, 31);
+        }
+    }
+    __syncthreads();
+
+    const int total = seg_lo[n_seg];
+    const int chunk = (total + a.n_splits - 1) / a.n_splits;
+    const int lo = min(split * chunk, total), hi = min(lo + chunk, total);
+    // ROPE: the newest tail row (the last key of the sequence, when there is a tail) is still unrotated
+    const int j_new = (ROPE && seg_lo[n_seg] > seg_lo[n_seg - 1]) ? total - 1 : -1;
+
+    const int g = threadIdx.x / LPK, sub = threadIdx.x % LPK;
+    // rotates the N elements this lane holds of a D-vector spread over LPK lanes
+    auto rotate = [&](float (&f)[N]) {
+        if (rope_pairing == SP_ROPE_HALF_SPLIT) {
+            const bool upper = sub >= LPK / 2;
+            const int m0 = (upper ? sub - LPK / 2 : sub) * N;
+#pragma unroll
+            for (int e = 0; e < N; ++e) {
+                const float other = __shfl_xor_sync(0xffffffffu, f[e], LPK / 2);
+                const float2 w = cs[m0 + e];
+                f[e] = upper ? fmaf(other, w.y, f[e] * w.x) : fmaf(-other, w.y, f[e] * w.x);
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < N; e += 2) {
+                const float2 w = cs[(sub * N + e) >> 1];
+                const float x0 = f[e], x1 = f[e + 1];
+                f[e] = x0 * w.x - x1 * w.y;
+                f[e + 1] = x0 * w.y + x1 * w.x;
+            }
+        }
+    };
+
+    float qf[GRP][N];
+#pragma unroll
+    for (int r = 0; r < GRP; ++r) {
+        Vec<T>::load(static_cast<const T *>(a.q) + ((int64_t)b * a.n_heads + h0 + r) * D + sub * N, qf[r]);
+        if (ROPE) {
+            rotate(qf[r]);
+#pragma unroll
+            for (int e = 0; e < N; ++e) qf[r][e] = to_float(T(qf[r][e]));   // the rounding a stored rotated query has
+        }
+#pragma unroll
+        for (int e = 0; e < N; ++e) qf[r][e] *= a.scale_log2e;
+    }
+
+    float m[GRP], l[GRP], acc[GRP][N];
+#pragma unroll
+    for (int r = 0; r < GRP; ++r) {
+        m[r] = -INFINITY; l[r] = 0.f;
+#pragma unroll
+        for (int e = 0; e < N; ++e) acc[r][e] = 0.f;
+    }
+    const float q_pos = ALIBI ? a.q_pos[b] : 0.f;
+    float slope_l2[GRP];
+#pragma unroll
+    for (int r = 0; r < GRP; ++r) slope_l2[r] = ALIBI ? a.slopes[h0 + r] * kLog2eD : 0.f;
+
+    int seg = 0;
+    for (int base = lo; base < hi; base += G * kDecUnroll) {   // trip count is block-uniform
+        uint4 kr[kDecUnroll], vr[kDecUnroll];
+        float kpos[kDecUnroll];
+        bool live[kDecUnroll];
+#pragma unroll
+        for (int u = 0; u < kDecUnroll; ++u) {                  // all loads of the batch first
+            const int j = base + g + u * G;
+            live[u] = j < hi;
+            if (live[u]) {
+                while (j >= seg_lo[seg + 1]) ++seg;             // keys ascend: segments only advance
+                const int64_t off = (int64_t)(j - seg_lo[seg]) * row_elems + sub * N;
+                kr[u] = ld_stream16(seg_k[seg] + off);
+                vr[u] = ld_stream16(seg_v[seg] + off);
+                if (ALIBI) kpos[u] = seg_pos[seg][j - seg_lo[seg]];
+            }
+        }
+        float s[GRP][kDecUnroll], cm[GRP];
+#pragma unroll
+        for (int r = 0; r < GRP; ++r) cm[r] = -INFINITY;
+        // ROPE: only the batch that holds the newest key (block-uniform test) takes the rotation path
+        const bool new_here = ROPE && j_new >= base && j_new < base + G * kDecUnroll;
+#pragma unroll
+        for (int u = 0; u < kDecUnroll; ++u) {
+            float kf[N];
+            if (live[u]) Raw16<T>::unpack(kr[u], kf);
+            if (ROPE && new_here) {
+                const bool is_new = live[u] && base + g + u * G == j_new;
+                if (__any_sync(0xffffffffu, is_new)) {           // once per (prompt, KV head): rotate the new key
+                    float rf[N];
+#pragma unroll
+                    for (int e = 0; e < N; ++e) rf[e] = live[u] ? kf[e] : 0.f;
+                    rotate(rf);
+                    if (is_new) {
+                        T *dst = const_cast<T *>(seg_k[n_seg - 1]) + (int64_t)(j_new - seg_lo[n_seg - 1]) * row_elems + sub * N;
+#pragma unroll
+                        for (int e = 0; e < N; ++e) { store_val(dst + e, rf[e]); kf[e] = to_float(T(rf[e])); }
+                    }
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < GRP; ++r) {
+                float d = 0.f;
+                if (live[u]) {
+#pragma unroll
+                    for (int e = 0; e < N; ++e) d = fmaf(qf[r][e], kf[e], d);
+                }
+#pragma unroll
+                for (int o = LPK / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+                if (ALIBI && live[u]) d -= slope_l2[r] * fabsf(q_pos - kpos[u]);
+                s[r][u] = live[u] ? d : -INFINITY;
+                cm[r] = fmaxf(cm[r], s[r][u]);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < GRP; ++r) {
+            if (cm[r] > m[r]) {
+                const float sc = ex2f(m[r] - cm[r]);
+                l[r] *= sc;
+#pragma unroll
+                for (int e = 0; e < N; ++e) acc[r][e] *= sc;
+                m[r] = cm[r];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kDecUnroll; ++u) {
+            if (live[u]) {
+                float vf[N];
+                Raw16<T>::unpack(vr[u], vf);
+#pragma unroll
+                for (int r = 0; r < GRP; ++r) {
+                    const float p = ex2f(s[r][u] - m[r]);
+                    l[r] += p;
+#pragma unroll
+                    for (int e = 0; e < N; ++e) acc[r][e] = fmaf(p, vf[e], acc[r][e]);
+                }
+            }
+        }
+    }
+
+    // ---- combine the key groups of this block (fixed order) ---------------------------
+#pragma unroll
+    for (int r = 0; r < GRP; ++r) {
+        float *mine = red + (g * GRP + r) * PS;
+#pragma unroll
+        for (int e = 0; e < N; ++e) mine[sub * N + e] = acc[r][e];
+        if (sub == 0) { mine[D] = m[r]; mine[D + 1] = l[r]; }
+    }
+    __syncthreads();
+
+    float bm[GRP], bl[GRP], bo[GRP];
+#pragma unroll
+    for (int r = 0; r < GRP; ++r) {
+        bm[r] = -INFINITY; bl[r] = 0.f; bo[r] = 0.f;
+        for (int i = 0; i < G; ++i) bm[r] = fmaxf(bm[r], red[(i * GRP + r) * PS + D]);
+        if (threadIdx.x < D) {
+            for (int i = 0; i < G; ++i) {
+                const float gm = red[(i * GRP + r) * PS + D];
+                const float w = (gm == -INFINITY) ? 0.f : ex2f(gm - bm[r]);
+                bl[r] += red[(i * GRP + r) * PS + D + 1] * w;
+                bo[r] += red[(i * GRP + r) * PS + threadIdx.x] * w;
+            }
+        }
+    }
+
+    if (a.n_splits > 1) {
+        // ---- merge the splits through the cluster's shared memory, in split order ---------
+        cg::cluster_group cluster = cg::this_cluster();
+        if (threadIdx.x < D) {
+#pragma unroll
+            for (int r = 0; r < GRP; ++r) {
+                part[r * PS + threadIdx.x] = bo[r];
+                if (threadIdx.x == 0) { part[r * PS + D] = bm[r]; part[r * PS + D + 1] = bl[r]; }
+            }
+        }
+        cluster.sync();
+        if (split == 0 && threadIdx.x < D) {
+#pragma unroll
+            for (int r = 0; r < GRP; ++r) {
+                float M = -INFINITY;
+                for (int i = 0; i < a.n_splits; ++i) M = fmaxf(M, cluster.map_shared_rank(part, i)[r * PS + D]);
+                float L = 0.f, O = 0.f;
+                for (int i = 0; i < a.n_splits; ++i) {
+                    const float *rp = cluster.map_shared_rank(part, i) + r * PS;
+                    const float w = (rp[D] == -INFINITY) ? 0.f : ex2f(rp[D] - M);
+                    L += rp[D + 1] * w;
+                    O += rp[threadIdx.x] * w;
+                }
+                bm[r] = M; bl[r] = L; bo[r] = O;
+            }
+        }
+        cluster.sync();                     // the others' shared memory stays alive until it has been read
+        if (split != 0) return;
+    }
+    if (threadIdx.x < D) {
+#pragma unroll
+        for (int r = 0; r < GRP; ++r) {
+            const int64_t bh = (int64_t)b * a.n_heads + h0 + r;
+            const float inv = bl[r] > 0.f ? 1.f / bl[r] : 0.f;
+            store_val(static_cast<T *>(a.out) + bh * D + threadIdx.x, bo[r] * inv);
+            if (threadIdx.x == 0 && a.lse) a.lse[bh] = bl[r] > 0.f ? (bm[r] + log2f(bl[r])) * kLn2D : -INFINITY;
+        }
+    }
+}
+
+// Splits of a launch: a power of two (cluster size), at most 16, such that one launch stays
+// within about one resident wave and a split keeps at least 32 keys.
+static int cluster_splits(int n_prompts, int blocks_y, int64_t max_keys, int blocks_per_sm)
+{
+    const int64_t by = std::max<int64_t>(1, (int64_t)n_prompts * blocks_y);
+    const int64_t want = std::min<int64_t>(((int64_t)blocks_per_sm * num_sms()) / by, (max_keys + 31) / 32);
+    int n = 1;
+    while (n * 2 <= want && n < 16) n *= 2;
+    return n;
+}
+
+template <typename T, int D, int GRP, bool ALIBI, bool ROPE>
+static int launch_decode_cluster(DecodeArgs a, const DecodeRope &rope, int pairing, int n_prompts, int64_t max_keys,
+                                 cudaStream_t st)
+{
+    constexpr int G = kDecThreads / (D / Vec<T>::N);
+    constexpr int PS = D + 2;
+    const int group = a.n_heads / a.n_kv_heads;
+    const int blocks_y = a.n_kv_heads * (group / GRP);
+    a.n_splits = cluster_splits(n_prompts, blocks_y, max_keys, GRP == 1 ? 8 : (GRP == 2 ? 5 : 3));
+    const int n_seg = a.k + 2;
+    const size_t smem = round_up((n_seg + 1) * sizeof(int), 16) + 3 * n_seg * sizeof(void *) +
+                        (size_t)(G + 1) * GRP * PS * sizeof(float) + (D / 2) * sizeof(float2);
+    SP_REQUIRE(smem <= 200 * 1024, SP_ERR_UNSUPPORTED, "sp_pruned_decode: k = %d needs too much shared memory", a.k);
+    auto kern = decode_cluster_kernel<T, D, GRP, ALIBI, ROPE>;
+    if (smem > 48 * 1024)
+        SP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if (a.n_splits > 8)
+        SP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.n_splits, blocks_y, n_prompts);
+    cfg.blockDim = dim3(kDecThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = a.n_splits; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = a.n_splits > 1 ? 1 : 0;      // one block per (prompt, KV head group): a plain launch
+    SP_CUDA(cudaLaunchKernelEx(&cfg, kern, a, rope, pairing));
+    return SP_OK;
+}
+
+template <typename T, int D, bool ALIBI, bool ROPE>
+static int launch_decode_grp(const DecodeArgs &a, const DecodeRope &rope, int pairing, int n_prompts, int64_t max_keys,
+                             cudaStream_t st)
+{
+    // query heads per block: the largest of 4, 2, 1 that divides the group, so grouped heads share
+    // one pass over their K and V rows
+    const int group = a.n_heads / a.n_kv_heads;
+    if (group % 4 == 0) return launch_decode_cluster<T, D, 4, ALIBI, ROPE>(a, rope, pairing, n_prompts, max_keys, st);
+    if (group % 2 == 0) return launch_decode_cluster<T, D, 2, ALIBI, ROPE>(a, rope, pairing, n_prompts, max_keys, st);
+    return launch_decode_cluster<T, D, 1, ALIBI, ROPE>(a, rope, pairing, n_prompts, max_keys, st);
+}
+
+template <bool ALIBI, bool ROPE>
+static int launch_decode_any(const DecodeArgs &a, const DecodeRope &rope, int pairing, int n_prompts, int64_t max_keys,
+                             int head_dim, int dtype, cudaStream_t st)
+{
+    if (dtype == SP_BF16)
+        return head_dim == 128 ? launch_decode_grp<__nv_bfloat16, 128, ALIBI, ROPE>(a, rope, pairing, n_prompts, max_keys, st)
+                               : launch_decode_grp<__nv_bfloat16, 64, ALIBI, ROPE>(a, rope, pairing, n_prompts, max_keys, st);
+    return head_dim == 128 ? launch_decode_grp<float, 128, ALIBI, ROPE>(a, rope, pairing, n_prompts, max_keys, st)
+                           : launch_decode_grp<float, 64, ALIBI, ROPE>(a, rope, pairing, n_prompts, max_keys, st);
+}
+
 }  // namespace sp
 
 extern "C" size_t sp_decode_workspace_bytes(int n_prompts, int n_heads, int head_dim)
@@ -294,9 +656,9 @@ static int decode_with_workspace(const void *q, const void *k_cache, const void 
                                  const sp_layout *lay, const int32_t *kept_idx, int k,
                                  const void *tail_k, const void *tail_v, const int32_t *tail_len,
                                  int tail_cap, int64_t max_keys, const float *q_pos, const float *cache_pos,
-                                 const float *tail_pos, const float *slopes, int n_heads, int n_kv_heads,
-                                 int head_dim, float scale, void *out, float *lse, void *ws,
-                                 size_t ws_bytes, int dtype, void *stream)
+                                 const float *tail_pos, const float *slopes, double rope_base, int pairing,
+                                 int n_heads, int n_kv_heads, int head_dim, float scale, void *out, float *lse,
+                                 void *ws, size_t ws_bytes, bool ws_required, int dtype, void *stream)
 {
     SP_REQUIRE(dtype == SP_F32 || dtype == SP_BF16, SP_ERR_INVALID_ARG, "sp_pruned_decode: unknown dtype %d", dtype);
     if (int rc = check_layout(lay)) return rc;
@@ -315,34 +677,37 @@ static int decode_with_workspace(const void *q, const void *k_cache, const void 
     SP_REQUIRE(aligned16(q) && aligned16(out) && aligned16(k_cache) && aligned16(v_cache) &&
                    aligned16(tail_k) && aligned16(tail_v),
                SP_ERR_INVALID_ARG, "sp_pruned_decode: data pointers must be 16-byte aligned");
-    SP_REQUIRE(ws && aligned256(ws) && ws_bytes >= sp_decode_workspace_bytes(lay->n_prompts, n_heads, head_dim),
-               SP_ERR_WORKSPACE, "sp_pruned_decode: workspace of %zu bytes (256-byte aligned) required",
-               sp_decode_workspace_bytes(lay->n_prompts, n_heads, head_dim));
+    if (ws_required)
+        SP_REQUIRE(ws && aligned256(ws) && ws_bytes >= sp_decode_workspace_bytes(lay->n_prompts, n_heads, head_dim),
+                   SP_ERR_WORKSPACE, "sp_pruned_decode: workspace of %zu bytes (256-byte aligned) required",
+                   sp_decode_workspace_bytes(lay->n_prompts, n_heads, head_dim));
 
     if (max_keys == 0) max_keys = (int64_t)lay->max_pre_len + (int64_t)k * lay->max_path_len + tail_cap;
-    const int cap = decode_split_cap(lay->n_prompts, n_heads);
-    const int n_splits = (int)std::max<int64_t>(1, std::min<int64_t>(cap, (max_keys + 31) / 32));
-
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t cbytes = decode_counter_bytes(lay->n_prompts, n_heads);
-    SP_CUDA(cudaMemsetAsync(ws, 0, 256 + cbytes, st));      // status word + split counters
 
+    // The cluster kernel needs no scratch: the workspace is accepted (and checked) for the sake of
+    // the interface, and its status word is left alone (this call has no bounded waits).
     DecodeArgs a;
     a.q = q; a.k_cache = k_cache; a.v_cache = v_cache; a.tail_k = tail_k; a.tail_v = tail_v;
     a.ppo = lay->prompt_path_off; a.pre_start = lay->pre_start; a.pre_len = lay->pre_len;
     a.path_start = lay->path_start; a.doc_len = lay->doc_len; a.qry_len = lay->qry_len;
     a.kept_idx = kept_idx; a.tail_len = tail_len; a.out = out; a.lse = lse;
-    a.counters = reinterpret_cast<unsigned int *>(static_cast<char *>(ws) + 256);
-    a.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + 256 + cbytes);
+    a.counters = nullptr; a.partial = nullptr;
     a.k = k; a.tail_cap = tail_cap; a.n_heads = n_heads; a.n_kv_heads = n_kv_heads;
-    a.n_splits = n_splits; a.scale_log2e = scale * kLog2eD;
+    a.n_splits = 1; a.scale_log2e = scale * kLog2eD;
     a.q_pos = q_pos; a.cache_pos = cache_pos; a.tail_pos = tail_pos; a.slopes = slopes;
 
-    if (dtype == SP_BF16)
-        return head_dim == 128 ? launch_decode<__nv_bfloat16, 128>(a, lay->n_prompts, st)
-                               : launch_decode<__nv_bfloat16, 64>(a, lay->n_prompts, st);
-    return head_dim == 128 ? launch_decode<float, 128>(a, lay->n_prompts, st)
-                           : launch_decode<float, 64>(a, lay->n_prompts, st);
+    DecodeRope rope = {};
+    if (rope_base > 0.0) {
+        SP_REQUIRE(slopes == nullptr, SP_ERR_INVALID_ARG, "sp_pruned_decode: rotary and ALiBi variants exclude each other");
+        const int group = n_heads / n_kv_heads;
+        SP_REQUIRE(group == 1 || group == 2 || group == 4, SP_ERR_UNSUPPORTED,
+                   "sp_pruned_decode_rope: %d query heads per KV head (1, 2 or 4 supported: one block must own the new key)", group);
+        for (int m = 0; m < head_dim / 2; ++m) rope.inv_freq[m] = std::pow(rope_base, -2.0 * m / head_dim);
+        return launch_decode_any<false, true>(a, rope, pairing, lay->n_prompts, max_keys, head_dim, dtype, st);
+    }
+    return slopes ? launch_decode_any<true, false>(a, rope, 0, lay->n_prompts, max_keys, head_dim, dtype, st)
+                  : launch_decode_any<false, false>(a, rope, 0, lay->n_prompts, max_keys, head_dim, dtype, st);
 }
 }  // namespace sp
 
@@ -354,8 +719,8 @@ extern "C" int sp_pruned_decode(const void *q, const void *k_cache, const void *
                                 size_t ws_bytes, int dtype, void *stream)
 {
     return sp::decode_with_workspace(q, k_cache, v_cache, lay, kept_idx, k, tail_k, tail_v, tail_len, tail_cap,
-                                     max_keys, nullptr, nullptr, nullptr, nullptr, n_heads, n_kv_heads, head_dim,
-                                     scale, out, lse, ws, ws_bytes, dtype, stream);
+                                     max_keys, nullptr, nullptr, nullptr, nullptr, 0.0, 0, n_heads, n_kv_heads, head_dim,
+                                     scale, out, lse, ws, ws_bytes, true, dtype, stream);
 }
 
 extern "C" int sp_pruned_decode_alibi(const void *q, const void *k_cache, const void *v_cache,
@@ -370,8 +735,24 @@ extern "C" int sp_pruned_decode_alibi(const void *q, const void *k_cache, const 
     SP_REQUIRE(lay == nullptr || lay->n_prompts == 0 || (q_pos && cache_pos && slopes && (tail_cap == 0 || tail_pos)),
                SP_ERR_INVALID_ARG, "sp_pruned_decode_alibi: q_pos, cache_pos, slopes (and tail_pos with a tail) are required");
     return decode_with_workspace(q, k_cache, v_cache, lay, kept_idx, k, tail_k, tail_v, tail_len, tail_cap, max_keys,
-                                 q_pos, cache_pos, tail_pos, slopes, n_heads, n_kv_heads, head_dim, scale, out,
-                                 lse, ws, ws_bytes, dtype, stream);
+                                 q_pos, cache_pos, tail_pos, slopes, 0.0, 0, n_heads, n_kv_heads, head_dim, scale, out,
+                                 lse, ws, ws_bytes, true, dtype, stream);
+}
+
+extern "C" int sp_pruned_decode_rope(const void *q, const void *k_cache, const void *v_cache,
+                                     const sp_layout *lay, const int32_t *kept_idx, int k, void *tail_k,
+                                     const void *tail_v, const int32_t *tail_len, int tail_cap, int64_t max_keys,
+                                     const float *q_pos, double rope_base, int pairing, int n_heads, int n_kv_heads,
+                                     int head_dim, float scale, void *out, float *lse, int dtype, void *stream)
+{
+    using namespace sp;
+    SP_REQUIRE(rope_base > 0.0, SP_ERR_INVALID_ARG, "sp_pruned_decode_rope: base must be positive");
+    SP_REQUIRE(pairing == SP_ROPE_HALF_SPLIT || pairing == SP_ROPE_INTERLEAVED, SP_ERR_INVALID_ARG,
+               "sp_pruned_decode_rope: unknown pairing %d", pairing);
+    SP_REQUIRE(lay == nullptr || lay->n_prompts == 0 || q_pos, SP_ERR_INVALID_ARG, "sp_pruned_decode_rope: q_pos is NULL");
+    return decode_with_workspace(q, k_cache, v_cache, lay, kept_idx, k, tail_k, tail_v, tail_len, tail_cap, max_keys,
+                                 q_pos, nullptr, nullptr, nullptr, rope_base, pairing, n_heads, n_kv_heads, head_dim,
+                                 scale, out, lse, nullptr, 0, false, dtype, stream);
 }
 
 // ---------------------------------------------------------------------------------------

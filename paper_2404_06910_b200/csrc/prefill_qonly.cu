@@ -360,7 +360,7 @@ int launch_prefill_qonly(const void *q, const void *k, const void *v, const sp_l
     p.total_tokens = lay->total_tokens; p.scale_log2e = scale * kLog2eQ;
     p.pos = pos; p.slopes = slopes;
     const int smem = (2 * kQStages + 1) * kTileB;
-    const int grid = (int)std::min<int64_t>(items, (int64_t)kQBlocksPerSM * kNumSMs);
+    const int grid = (int)std::min<int64_t>(items, (int64_t)kQBlocksPerSM * num_sms());
     if (pos) {
         SP_CUDA(cudaFuncSetAttribute(prefill_qonly_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         prefill_qonly_kernel<true><<<grid, kQThreads, smem, st>>>(p);

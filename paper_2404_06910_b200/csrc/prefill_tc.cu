@@ -613,7 +613,7 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
 
     const int64_t items = max_tiles(lay->n_prompts, lay->n_paths, lay->max_pre_len, lay->max_path_len) * n_heads;
     if (items == 0) return SP_OK;
-    const int grid = (int)std::min<int64_t>(items, 2 * kNumSMs);
+    const int grid = (int)std::min<int64_t>(items, 2 * num_sms());
     const int smem = kQBytes + 4 * kKVBytes + 4 * 2048 + 1024;
     if (pos) {
         SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));

@@ -147,7 +147,7 @@ static int launch_rope(void *x, void *x1, const float *pos, int64_t n_tokens, in
     const bool v0 = rope_vec_ok<T>(x, ld_token, head_dim, rot_dim, pairing);
     const bool v1 = x1 == nullptr || rope_vec_ok<T>(x1, ld_token1, head_dim, rot_dim, pairing);
     const int64_t n_groups = (n_tokens + kRopeTokens - 1) / kRopeTokens;
-    const int grid = (int)std::min<int64_t>(n_groups, (int64_t)kNumSMs * 16);
+    const int grid = (int)std::min<int64_t>(n_groups, (int64_t)num_sms() * 16);
     auto go = [&](auto kern) {
         kern<<<grid, kRopeThreads, 0, st>>>((T *)x, (T *)x1, pos, n_tokens, ld_token, ld_token1, n_heads, n_heads1,
                                             head_dim, rot_dim, pairing, fr);

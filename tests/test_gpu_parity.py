@@ -661,3 +661,78 @@ def test_decode_alibi_parity(dtype, D):
     sp.sp_check_status(ws)
     assert rel_l2(f32(out), ref_o) <= TOL[dtype]
     np.testing.assert_allclose(lse.cpu().numpy(), ref_l, atol=2e-5 if dtype == "f32" else 2e-2)
+
+
+# ------------------------------------------------------------------------- decode with the rotation folded in
+@pytest.mark.parametrize("dtype,D", [("f32", 64), ("f32", 128), ("bf16", 64), ("bf16", 128)])
+@pytest.mark.parametrize("pairing", [0, 1])
+@pytest.mark.parametrize("H,Hkv", [(4, 4), (4, 2), (8, 2)])
+def test_decode_rope_fused(dtype, D, pairing, H, Hkv):
+    """sp_pruned_decode_rope against the oracle's rope followed by its decode, over three steps
+    (so that keys rotated and written back by earlier steps are read again), and the stored
+    tail keys against the stand-alone rotation."""
+    lay = build_layout([16, 3, 0], [[32, 1, 129, 40], [200, 17], [5]], [[8, 8, 8, 8], [5, 5], [2]])
+    B, T, cap, k = lay.n_prompts, lay.total_tokens, 4, 2
+    kc, vc = _randn((T, Hkv, D), dtype, 700), _randn((T, Hkv, D), dtype, 701)
+    tk, tv = _randn((B, cap, Hkv, D), dtype, 703), _randn((B, cap, Hkv, D), dtype, 704)
+    kept = np.array([[2, 0], [4, -1], [-1, -1]], np.int32)
+    dl = sp.DeviceLayout.from_host(lay)
+    scale = 1 / math.sqrt(D)
+    rnd = (lambda a: a) if dtype == "f32" else (lambda a: torch.from_numpy(a).bfloat16().float().numpy())
+    tkd, kcd, vcd, tvd, keptd = dev(tk), dev(kc), dev(vc), dev(tv), dev(kept)
+    tk_ref = f32(tk).copy()                                   # oracle's tail: rows rotated as the steps go
+    tk_sep = dev(tk)                                          # rotated by the stand-alone kernel
+    for step in range(3):
+        q = _randn((B, H, D), dtype, 710 + step)
+        pos = np.array([301.25 + step, 17.5 + 2 * step, 3.0 + step], np.float32)
+        tl = np.array([step + 1, step + 1, step + 1 if step else 0], np.int32)   # prompt 2 has no tail at step 0
+        out = torch.full((B, H, D), float("nan"), dtype=TDT[dtype], device="cuda")
+        lse = torch.full((B, H), float("nan"), device="cuda")
+        sp.sp_pruned_decode_rope(dev(q), kcd, vcd, dl, keptd, k, tkd, tvd, dev(tl), cap, dev(pos), scale, out, lse,
+                                 pairing=pairing)
+        torch.cuda.synchronize()
+        # oracle: rotate q and each prompt's newest tail row, then decode
+        q_ref = rnd(oracle.rope(f32(q), pos, pairing=pairing))
+        for b in range(B):
+            if tl[b] > 0:
+                r = tl[b] - 1
+                tk_ref[b, r] = rnd(oracle.rope(np.ascontiguousarray(tk_ref[b, r][None]), pos[b:b + 1], pairing=pairing))[0]
+                sp.sp_rope_apply(tk_sep[b, r], dev(pos[b:b + 1]), Hkv, D, n_tokens=1, pairing=pairing)
+        ref_o, ref_l = oracle.pruned_decode(q_ref, f32(kc), f32(vc), lay, kept, tk_ref, f32(tv), tl, scale)
+        assert rel_l2(f32(out), ref_o) <= TOL[dtype]
+        fin = np.isfinite(ref_l)
+        np.testing.assert_allclose(lse.cpu().numpy()[fin], ref_l[fin], atol=1e-5 if dtype == "f32" else 2e-2)
+        # the rows written back: what the stand-alone rotation stores, up to one rounding of the last place
+        got_t, sep_t = f32(tkd), f32(tk_sep)
+        for b in range(B):
+            rows = slice(0, int(tl[b]))
+            tol = 2e-6 if dtype == "f32" else 2.0 ** -7
+            assert np.all(np.abs(got_t[b, rows] - sep_t[b, rows]) <= np.abs(sep_t[b, rows]) * tol + 2e-6)
+            np.testing.assert_array_equal(got_t[b, int(tl[b]):], f32(tk)[b, int(tl[b]):])    # later rows untouched
+
+
+def test_decode_rope_rejects_wide_groups():
+    lay = build_layout([4], [[8]], [[2]])
+    dl = sp.DeviceLayout.from_host(lay)
+    q = dev(_randn((1, 8, 64), "f32", 1))
+    kc = dev(_randn((lay.total_tokens, 1, 64), "f32", 2))
+    tk = dev(_randn((1, 1, 1, 64), "f32", 3))
+    with pytest.raises(sp.SpError) as e:
+        sp.sp_pruned_decode_rope(q, kc, kc, dl, dev(np.array([[0]], np.int32)), 1, tk, tk, dev(np.array([1], np.int32)), 1,
+                                 dev(np.array([5.0], np.float32)), 0.125, torch.empty_like(q))
+    assert e.value.code == sp.SP_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("H,Hkv", [(8, 1), (8, 2), (6, 3), (6, 2), (3, 1), (32, 8)])
+def test_decode_grouped_heads(H, Hkv):
+    """Query heads that share a KV head are served by one block per group of 4, 2 or 1 heads."""
+    lay = build_layout([16, 3], [[32, 1, 129, 40], [200, 17]], [[8, 8, 8, 8], [5, 5]])
+    _decode_case(lay, H, Hkv, 128, "bf16", 2, [[2, 0], [4, -1]], 6, [6, 1], 540)
+    _decode_case(lay, H, Hkv, 64, "f32", 2, [[3, 1], [5, 4]], 2, [0, 2], 541)
+
+
+def test_decode_long_sequences_many_splits():
+    """Few (prompt, head) pairs and thousands of keys: the largest cluster (16 blocks) and many loop trips."""
+    lay = build_layout([64], [[2000, 1500, 3000]], [[32, 32, 32]])
+    _decode_case(lay, 2, 2, 128, "bf16", 3, [[2, 0, 1]], 40, [37], 550)
+    _decode_case(lay, 1, 1, 64, "f32", 2, [[1, 2]], 8, [8], 551)
