@@ -294,8 +294,11 @@ struct DecodeRope {
     double inv_freq[64];      // base^(-2m/D), m < D/2 <= 64
 };
 
-template <typename T, int D, int GRP, bool ALIBI, bool ROPE>
-__global__ void __launch_bounds__(kDecThreads, GRP == 1 ? 8 : (GRP == 2 ? 5 : 3))
+// MINB: resident blocks per SM the register budget is sized for.  Split launches want 8 (a whole
+// launch in one wave, clusters of 2^n blocks pack evenly); an unsplit launch over a large batch
+// runs faster with the few registers more that 7 leave (nothing spills).
+template <typename T, int D, int GRP, bool ALIBI, bool ROPE, int MINB>
+__global__ void __launch_bounds__(kDecThreads, MINB)
 decode_cluster_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ DecodeRope rope, int rope_pairing)
 {
     namespace cg = cooperative_groups;
@@ -380,6 +383,8 @@ decode_cluster_kernel(const __grid_constant__ DecodeArgs a, const __grid_constan
     const int lo = min(split * chunk, total), hi = min(lo + chunk, total);
     // ROPE: the newest tail row (the last key of the sequence, when there is a tail) is still unrotated
     const int j_new = (ROPE && seg_lo[n_seg] > seg_lo[n_seg - 1]) ? total - 1 : -1;
+    const bool owns_new = j_new >= lo && j_new < hi;                 // block-uniform; j_new is then hi - 1
+    const int hi_loop = owns_new ? hi - 1 : hi;                        // the new key is handled after the loop
 
     const int g = threadIdx.x / LPK, sub = threadIdx.x % LPK;
     // rotates the N elements this lane holds of a D-vector spread over LPK lanes
@@ -430,14 +435,14 @@ decode_cluster_kernel(const __grid_constant__ DecodeArgs a, const __grid_constan
     for (int r = 0; r < GRP; ++r) slope_l2[r] = ALIBI ? a.slopes[h0 + r] * kLog2eD : 0.f;
 
     int seg = 0;
-    for (int base = lo; base < hi; base += G * kDecUnroll) {   // trip count is block-uniform
+    for (int base = lo; base < hi_loop; base += G * kDecUnroll) {   // trip count is block-uniform
         uint4 kr[kDecUnroll], vr[kDecUnroll];
         float kpos[kDecUnroll];
         bool live[kDecUnroll];
 #pragma unroll
         for (int u = 0; u < kDecUnroll; ++u) {                  // all loads of the batch first
             const int j = base + g + u * G;
-            live[u] = j < hi;
+            live[u] = j < hi_loop;
             if (live[u]) {
                 while (j >= seg_lo[seg + 1]) ++seg;             // keys ascend: segments only advance
                 const int64_t off = (int64_t)(j - seg_lo[seg]) * row_elems + sub * N;
@@ -449,26 +454,10 @@ decode_cluster_kernel(const __grid_constant__ DecodeArgs a, const __grid_constan
         float s[GRP][kDecUnroll], cm[GRP];
 #pragma unroll
         for (int r = 0; r < GRP; ++r) cm[r] = -INFINITY;
-        // ROPE: only the batch that holds the newest key (block-uniform test) takes the rotation path
-        const bool new_here = ROPE && j_new >= base && j_new < base + G * kDecUnroll;
 #pragma unroll
         for (int u = 0; u < kDecUnroll; ++u) {
             float kf[N];
             if (live[u]) Raw16<T>::unpack(kr[u], kf);
-            if (ROPE && new_here) {
-                const bool is_new = live[u] && base + g + u * G == j_new;
-                if (__any_sync(0xffffffffu, is_new)) {           // once per (prompt, KV head): rotate the new key
-                    float rf[N];
-#pragma unroll
-                    for (int e = 0; e < N; ++e) rf[e] = live[u] ? kf[e] : 0.f;
-                    rotate(rf);
-                    if (is_new) {
-                        T *dst = const_cast<T *>(seg_k[n_seg - 1]) + (int64_t)(j_new - seg_lo[n_seg - 1]) * row_elems + sub * N;
-#pragma unroll
-                        for (int e = 0; e < N; ++e) { store_val(dst + e, rf[e]); kf[e] = to_float(T(rf[e])); }
-                    }
-                }
-            }
 #pragma unroll
             for (int r = 0; r < GRP; ++r) {
                 float d = 0.f;
@@ -505,6 +494,45 @@ decode_cluster_kernel(const __grid_constant__ DecodeArgs a, const __grid_constan
 #pragma unroll
                     for (int e = 0; e < N; ++e) acc[r][e] = fmaf(p, vf[e], acc[r][e]);
                 }
+            }
+        }
+    }
+
+    if (ROPE && owns_new && threadIdx.x < 32) {
+        // The newest key, outside the streaming loop: warp 0 loads the unrotated row (every key
+        // group of the warp holds a copy), rotates it, group 0 writes it back for the later steps
+        // and takes it into its running softmax like any other key.
+        const int64_t off = (int64_t)(j_new - seg_lo[n_seg - 1]) * row_elems + sub * N;
+        T *krow = const_cast<T *>(seg_k[n_seg - 1]) + off;
+        float kf[N], vf[N];
+        Vec<T>::load(krow, kf);
+        Vec<T>::load(seg_v[n_seg - 1] + off, vf);
+        rotate(kf);
+#pragma unroll
+        for (int e = 0; e < N; ++e) kf[e] = to_float(T(kf[e]));           // as it is stored
+        if (g == 0) {
+#pragma unroll
+            for (int e = 0; e < N; ++e) store_val(krow + e, kf[e]);
+        }
+#pragma unroll
+        for (int r = 0; r < GRP; ++r) {
+            float d = 0.f;
+#pragma unroll
+            for (int e = 0; e < N; ++e) d = fmaf(qf[r][e], kf[e], d);
+#pragma unroll
+            for (int o = LPK / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+            if (g == 0) {
+                if (d > m[r]) {
+                    const float sc = ex2f(m[r] - d);
+                    l[r] *= sc;
+#pragma unroll
+                    for (int e = 0; e < N; ++e) acc[r][e] *= sc;
+                    m[r] = d;
+                }
+                const float p = ex2f(d - m[r]);
+                l[r] += p;
+#pragma unroll
+                for (int e = 0; e < N; ++e) acc[r][e] = fmaf(p, vf[e], acc[r][e]);
             }
         }
     }
@@ -593,12 +621,14 @@ static int launch_decode_cluster(DecodeArgs a, const DecodeRope &rope, int pairi
     constexpr int PS = D + 2;
     const int group = a.n_heads / a.n_kv_heads;
     const int blocks_y = a.n_kv_heads * (group / GRP);
-    a.n_splits = cluster_splits(n_prompts, blocks_y, max_keys, GRP == 1 ? 8 : (GRP == 2 ? 5 : 3));
+    constexpr int kMinB = GRP == 1 ? 8 : (GRP == 2 ? 5 : 3);
+    a.n_splits = cluster_splits(n_prompts, blocks_y, max_keys, kMinB);
     const int n_seg = a.k + 2;
     const size_t smem = round_up((n_seg + 1) * sizeof(int), 16) + 3 * n_seg * sizeof(void *) +
                         (size_t)(G + 1) * GRP * PS * sizeof(float) + (D / 2) * sizeof(float2);
     SP_REQUIRE(smem <= 200 * 1024, SP_ERR_UNSUPPORTED, "sp_pruned_decode: k = %d needs too much shared memory", a.k);
-    auto kern = decode_cluster_kernel<T, D, GRP, ALIBI, ROPE>;
+    auto kern = (GRP == 1 && a.n_splits == 1) ? decode_cluster_kernel<T, D, GRP, ALIBI, ROPE, kMinB - (GRP == 1 ? 1 : 0)>
+                                              : decode_cluster_kernel<T, D, GRP, ALIBI, ROPE, kMinB>;
     if (smem > 48 * 1024)
         SP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     if (a.n_splits > 8)
