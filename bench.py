@@ -3,14 +3,19 @@
 
 One "step" is one pass of the whole path over one batch of synthetic prompts:
   RoPE(Q), RoPE(K) -> fork-join prefill -> path scores -> top-k -> decode_steps x
-  (RoPE of the new q and k rows, pruned decode).
+  (pruned decode with the rotation of the new q and k rows folded in).
 `value` is the prefill's useful TFLOP/s counted over the WHOLE step time (inputs resident
-in HBM); the per-kernel rates and roofline fractions are reported beside it.
+in HBM); `roofline` describes the prefill kernel (the one the metric is named after),
+`roofline_decode` the decode kernel, `kernels` every stage; times are medians over the timed
+steps.  After the default workload (cfg2) the two other large single-GPU workloads (cfg3,
+cfg4) are measured in the same process and reported under `workloads`.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
 
-N > 1 (torchrun): every rank runs its own batch (independent prompts, no data-path
-collective); the time is the max over ranks and `value` the aggregate ("weak" scaling).
+N > 1: started as a plain script, bench.py starts N ranks of itself (torch.distributed.run on
+127.0.0.1); started by torchrun it uses the ranks it is given.  Every rank runs its own batch
+(independent prompts, no data-path collective); the time is the max over ranks and `value`
+the aggregate ("weak" scaling).
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
 """
 from __future__ import annotations
@@ -36,12 +41,11 @@ from workloads import (draw_decode_inputs, draw_lengths, draw_logits, draw_prior
 METRIC = "superposition prefill useful TFLOP/s over the whole hot-path step"
 UNIT = "TFLOP/s"
 PREFILL_LAUNCHES = 2           # kernels sp_superpose_prefill launches per call (tile plan + attention)
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch, (kernel, workload) -> bytes, from
-# the ncu captures summarised under profiles/ (absent = not captured for the current kernel).
-NCU_TRAFFIC_BYTES = {
-    # scaled by tokens / prompts from the 20-prompt captures (traffic grows in proportion)
-    ("prefill", "cfg2_batched_serving"): 9.077e9,
-    ("decode", "cfg2_batched_serving"): 4.389e8,
+# dram__bytes_read.sum + dram__bytes_write.sum from the ncu captures summarised under profiles/,
+# per unit of work (the captures run a smaller case; traffic grows in proportion to the units).
+# Each entry names the hash of the kernel sources it was taken from: after a kernel change the
+# figure is withheld (null in the JSON line) until the capture is repeated.
+NCU_TRAFFIC = {
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -197,9 +201,9 @@ class HotPath:
         self.bytes_decode = None        # needs the kept set: filled after the first step
         # kernels launched per step (ours): rope x2, prefill, row_logp + path_sum, top-k,
         # per decode step rope (q and the new key in one launch) + decode
-        self.launches = 2 + PREFILL_LAUNCHES + 2 + 1 + self.steps_dec * 2
-        self.decode_graph = None
         self.fused_rope = (H // Hkv) in (1, 2, 4)
+        self.launches = 2 + PREFILL_LAUNCHES + 2 + 1 + self.steps_dec * (1 if self.fused_rope else 2)
+        self.decode_graph = None
         self.kv_sets = [(self.k, self.v)]
 
     def decode_bytes(self):
@@ -292,6 +296,202 @@ class HotPath:
 
 
 STAGES = ("rope", "prefill", "path_scores", "topk", "decode")
+PREFILL_SOURCES = ("prefill_tc.cu", "prefill_plan.cuh", "tc_ptx.cuh")
+DECODE_SOURCES = ("decode.cu",)
+
+
+def source_hash(names) -> str:
+    """Short hash of kernel source files: a captured ncu figure is only quoted while the kernel
+    it was taken from is unchanged."""
+    import hashlib
+    h = hashlib.sha256()
+    for n in names:
+        with open(os.path.join(ROOT, "paper_2404_06910_b200", "csrc", n), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
+
+
+def captured_traffic(kernel: str, workload: str, sources, units: float):
+    """dram bytes per launch from the ncu capture summarised under profiles/, scaled to this
+    launch by the units processed (tokens for the prefill, gathered keys for the decode);
+    None when there is no capture for this workload or the kernel changed since."""
+    ent = NCU_TRAFFIC.get((kernel, workload))
+    if ent is None or ent["source_hash"] != source_hash(sources):
+        return None, None
+    return ent["bytes_per_unit"] * units, (f"scaled by units from the capture of {ent['capture']} "
+                                           f"({ent['bytes_per_unit']:.1f} B per {ent['unit']})")
+
+
+def full_causal_pairs(lay) -> int:
+    """(query, key) pairs a plain causal mask over each prompt's packed rows would admit."""
+    tot = 0
+    for b in range(lay.n_prompts):
+        lo, hi = lay.prompt_row_range(b)
+        n = hi - lo
+        tot += n * (n + 1) // 2
+    return tot
+
+
+def measure_workload(cfg, sp, device, args, rank, dist, peaks, steps, warmup, with_e2e, l2_bytes):
+    """Times `steps` passes of the whole hot path on one workload; returns the per-kernel
+    figures (medians over the timed steps) and, for the rank's own use, the step time."""
+    hp = HotPath(cfg, rank_seed(cfg, rank), sp, device, args.prompts, args.decode_steps)
+    hp.make_kv_sets(l2_bytes)
+    if not args.no_graph:
+        hp.capture_decode_graph()
+    flush = None
+    if hp.bytes_prefill < 2 * l2_bytes:          # small workload: flush L2 between steps
+        flush = torch.empty(2 * l2_bytes, dtype=torch.uint8, device=device)
+
+    def sync():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        hp.step()
+        if flush is not None:
+            flush.zero_()
+    sync()
+    hp.bytes_decode = hp.decode_bytes()
+
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else 0)
+    if rank == 0:
+        sampler.start()
+    all_ev = []
+    sync()
+    for _ in range(steps):
+        ev = []
+        hp.step(ev)
+        all_ev.append(ev)
+        if flush is not None:
+            flush.zero_()
+    sync()
+    clocks = sampler.stop() if rank == 0 else None
+    per_step = np.array([[ev[i].elapsed_time(ev[i + 1]) for i in range(len(STAGES))] for ev in all_ev])
+    totals = np.array([ev[0].elapsed_time(ev[-1]) for ev in all_ev])
+    stage_ms = np.median(per_step, axis=0)
+    ms_per_step = float(np.median(totals))
+
+    def timed(fn, reps=5, per=1):
+        fn(); torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            if flush is not None:
+                flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) / per)
+        return float(np.median(ts))
+
+    def graph_of(fn):
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            fn()
+        return g
+
+    # decode kernel alone (no rotation of the new rows), replayed from a graph: the per-launch
+    # figure of that kernel; cold = KV sets rotate (as in the step), warm = one set re-read
+    n_dec = hp.steps_dec
+    dec_cold_ms = timed(graph_of(lambda: hp.decode_loop(with_rope=False)).replay, per=n_dec)
+    sets = hp.kv_sets
+    hp.kv_sets = sets[:1]
+    dec_warm_ms = timed(graph_of(lambda: hp.decode_loop(with_rope=False)).replay, per=n_dec)
+    hp.kv_sets = sets
+    # the decode step as an application without CUDA graphs would issue it: eager launches
+    dec_eager_ms = timed(lambda: hp.decode_loop(), reps=3, per=n_dec)
+
+    # cached / online mode of the prefill (only the query rows of every path are produced): timed
+    # on its own, it is not part of the step
+    qo_ms = None
+    if cfg.dtype == "bf16":
+        qo_ms = timed(lambda: sp.sp_superpose_prefill(hp.q, hp.k, hp.v, hp.dl, hp.scale, hp.out, None, hp.ws_pre,
+                                                      rows=sp.SP_ROWS_QUERY_ONLY))
+
+    # end to end: pinned host -> device copies of every input, the pass, device -> host results
+    e2e = None
+    if with_e2e:
+        e2e_steps = max(1, min(steps, 3))
+        hp.h2d(); hp.step(); hp.d2h(); sync()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e2e_steps):
+            bi = hp.h2d()
+            hp.step()
+            bo = hp.d2h()
+        e1.record()
+        sync()
+        e2e = {"ms": e0.elapsed_time(e1) / e2e_steps, "steps": e2e_steps, "h2d": bi, "d2h": bo}
+
+    tf = lambda flop, ms: flop / (ms * 1e-3) / 1e12
+    gb = lambda byt, ms: byt / (ms * 1e-3) / 1e9
+    ms = dict(zip(STAGES, (float(x) for x in stage_ms)))
+    hbm = peaks["hbm_gbs"]
+    pre_gbs, pre_tf = gb(hp.bytes_prefill, ms["prefill"]), tf(hp.flop_prefill, ms["prefill"])
+    ai = hp.flop_prefill / hp.bytes_prefill
+    bound_tf = min(peaks["bf16_tflops_sustained"], ai * hbm / 1e3)
+    dec_bytes = hp.bytes_decode / n_dec
+    kernels = {
+        "rope": {"ms": ms["rope"], "gbs": gb(hp.bytes_rope, ms["rope"]), "frac_hbm": gb(hp.bytes_rope, ms["rope"]) / hbm},
+        "prefill": {"ms": ms["prefill"], "useful_tflops": pre_tf, "gbs": pre_gbs,
+                    "frac_bf16_burst": pre_tf / peaks["bf16_tflops"],
+                    "frac_bf16_sustained": pre_tf / peaks["bf16_tflops_sustained"],
+                    "arith_intensity": ai, "binding_roofline_tflops": bound_tf, "frac_binding": pre_tf / bound_tf},
+        "path_scores": {"ms": ms["path_scores"], "gbs": gb(hp.bytes_scores, ms["path_scores"]),
+                        "frac_hbm": gb(hp.bytes_scores, ms["path_scores"]) / hbm},
+        "topk": {"ms": ms["topk"]},
+        "prefill_query_only": None if qo_ms is None else {
+            "ms": qo_ms, "useful_tflops": tf(hp.flop_query_only, qo_ms), "gbs": gb(hp.bytes_query_only, qo_ms),
+            "frac_hbm": gb(hp.bytes_query_only, qo_ms) / hbm,
+            "note": "SP_ROWS_QUERY_ONLY (cached preamble/doc KV, Algorithm 3's query batch); not part of the step"},
+        "decode": {"ms": ms["decode"], "steps": n_dec, "us_per_token": ms["decode"] / n_dec * 1e3,
+                   "gbs": gb(hp.bytes_decode, ms["decode"]), "frac_hbm": gb(hp.bytes_decode, ms["decode"]) / hbm,
+                   "kernel_only_us_cold": dec_cold_ms * 1e3, "kernel_only_frac_hbm_cold": gb(dec_bytes, dec_cold_ms) / hbm,
+                   "kernel_only_us_warm": dec_warm_ms * 1e3, "kernel_only_gbs_warm": gb(dec_bytes, dec_warm_ms),
+                   "ungraphed_us_per_token": dec_eager_ms * 1e3, "kv_sets": len(hp.kv_sets),
+                   "launches_per_token": 1 if hp.fused_rope else 2,
+                   "includes": ("one launch per token (the new query and key rows are rotated inside the decode kernel)"
+                                if hp.fused_rope else "1 rope launch (q and the new key) + 1 decode launch per token")
+                               + ("" if args.no_graph else ", replayed from a CUDA graph"),
+                   "warm_note": "warm = the same KV set re-read by every launch (may sit in L2): not compared with the HBM peak"},
+    }
+    T = hp.lay.total_tokens
+    keys_per_launch = dec_bytes / (2.0 * hp.Hkv * hp.D * cfg.elt_bytes)
+    tr_p, tr_p_note = captured_traffic("prefill", cfg.name, PREFILL_SOURCES, float(T))
+    tr_d, tr_d_note = captured_traffic("decode", cfg.name, DECODE_SOURCES, keys_per_launch)
+    roof_prefill = {"kernel": "prefill_tc_kernel (sp_superpose_prefill)", "bound": "hbm", "achieved": pre_gbs,
+                    "peak": hbm, "unit": "GB/s", "frac": pre_gbs / hbm, "traffic": tr_p, "traffic_note": tr_p_note,
+                    "peak_source": peaks["source"], "algorithmic_bytes": hp.bytes_prefill, "launch_ms": ms["prefill"],
+                    "useful_tflops": pre_tf, "frac_bf16_sustained": pre_tf / peaks["bf16_tflops_sustained"],
+                    "why_hbm": f"arithmetic intensity {ai:.1f} flop/B is below the ridge of the measured peaks"}
+    roof_decode = {"kernel": "decode_cluster_kernel (sp_pruned_decode)", "bound": "hbm", "achieved": gb(dec_bytes, dec_cold_ms),
+                   "peak": hbm, "unit": "GB/s", "frac": gb(dec_bytes, dec_cold_ms) / hbm, "traffic": tr_d,
+                   "traffic_note": tr_d_note, "peak_source": peaks["source"], "algorithmic_bytes": dec_bytes,
+                   "launch_ms": dec_cold_ms, "launches_per_step": n_dec}
+    res = {
+        "workload": cfg.name, "ms_per_step": ms_per_step, "steps": steps, "warmup": warmup,
+        "value": tf(hp.flop_prefill, ms_per_step), "frac_bf16_sustained": pre_tf / peaks["bf16_tflops_sustained"],
+        "config": {"workload": cfg.name, "prompts_per_gpu": hp.B, "paths": hp.lay.n_paths,
+                   "tokens": T, "heads": hp.H, "head_dim": hp.D, "vocab": cfg.vocab,
+                   "top_k": cfg.top_k, "decode_steps": n_dec, "allowed_pairs": hp.pairs,
+                   "decode_kv_sets": len(hp.kv_sets),
+                   "l2": "inputs larger than L2" if flush is None else "L2 flushed between steps",
+                   "timing": "median over the timed steps, CUDA events on the launching stream"},
+        "useful_vs_full_causal": hp.pairs / max(1, full_causal_pairs(hp.lay)),
+        "roofline": roof_prefill, "roofline_decode": roof_decode, "kernels": kernels,
+        "flop_prefill": hp.flop_prefill, "launches_per_step": hp.launches, "input_generation_s": hp.gen_s,
+        "clocks": clocks, "e2e": e2e,
+    }
+    del hp, flush
+    torch.cuda.empty_cache()
+    return res
 
 
 def run_ours(args):
@@ -307,157 +507,43 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
-    cfg = get_config(args.workload)
-    hp = HotPath(cfg, rank_seed(cfg, rank), sp, device, args.prompts, args.decode_steps)
-    l2_bytes = torch.cuda.get_device_properties(device).L2_cache_size
-    hp.make_kv_sets(l2_bytes)
-    if not args.no_graph:
-        hp.capture_decode_graph()
     peaks = load_peaks()
-    flush = None
-    if hp.bytes_prefill < 2 * l2_bytes:          # small workload: flush L2 between steps
-        flush = torch.empty(2 * l2_bytes, dtype=torch.uint8, device=device)
+    l2_bytes = torch.cuda.get_device_properties(device).L2_cache_size
+    cfg = get_config(args.workload)
+    main = measure_workload(cfg, sp, device, args, rank, dist, peaks, args.steps, args.warmup, not args.no_e2e, l2_bytes)
+    # the other large single-GPU workloads, in the same process: fewer steps, no host-copy leg
+    extra = []
+    if not args.no_extra and args.prompts is None and cfg.name.startswith("cfg2"):
+        for name in ("cfg3", "cfg4"):
+            extra.append(measure_workload(get_config(name), sp, device, args, rank, dist, peaks,
+                                          max(3, min(args.steps, 5)), 3, False, l2_bytes))
 
-    def sync():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(args.warmup):
-        hp.step()
-        if flush is not None:
-            flush.zero_()
-    sync()
-    hp.bytes_decode = hp.decode_bytes()
-
-    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else 0)
+    e2e_ms = main["e2e"]["ms"] if main["e2e"] else float("nan")
+    ms_per_step, e2e_ms = max_over_ranks([main["ms_per_step"], e2e_ms], dist, device)
     if rank == 0:
-        sampler.start()
-    all_ev = []
-    sync()
-    for _ in range(args.steps):
-        ev = []
-        hp.step(ev)
-        all_ev.append(ev)
-        if flush is not None:
-            flush.zero_()
-    sync()
-    clocks = sampler.stop() if rank == 0 else None
-
-    # decode kernel alone (no rope launches), eager, for the per-launch roofline of that kernel
-    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    hp.decode_loop(with_rope=False)
-    d0.record()
-    hp.decode_loop(with_rope=False)
-    d1.record()
-    sync()
-    decode_kernel_ms = d0.elapsed_time(d1) / hp.steps_dec
-
-    # cached / online mode of the prefill (only the query rows of every path are produced): timed
-    # on its own, it is not part of the step
-    qo_ms = None
-    if cfg.dtype == "bf16":
-        for _ in range(2):
-            sp.sp_superpose_prefill(hp.q, hp.k, hp.v, hp.dl, hp.scale, hp.out, None, hp.ws_pre, rows=sp.SP_ROWS_QUERY_ONLY)
-        ts = []
-        for _ in range(5):
-            if flush is not None:
-                flush.zero_()
-            q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            q0.record()
-            sp.sp_superpose_prefill(hp.q, hp.k, hp.v, hp.dl, hp.scale, hp.out, None, hp.ws_pre, rows=sp.SP_ROWS_QUERY_ONLY)
-            q1.record()
-            sync()
-            ts.append(q0.elapsed_time(q1))
-        qo_ms = float(np.median(ts))
-
-    stage_ms = np.zeros(len(STAGES))
-    total_ms = 0.0
-    for ev in all_ev:
-        for i in range(len(STAGES)):
-            stage_ms[i] += ev[i].elapsed_time(ev[i + 1])
-        total_ms += ev[0].elapsed_time(ev[-1])
-    stage_ms /= args.steps
-    ms_per_step = total_ms / args.steps
-
-    # end to end: pinned host -> device copies of every input, the pass, device -> host results
-    e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 3))
-    bi = bo = 0
-    e2e_ms = float("nan")
-    if e2e_steps:
-        hp.h2d(); hp.step(); hp.d2h(); sync()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(e2e_steps):
-            bi = hp.h2d()
-            hp.step()
-            bo = hp.d2h()
-        e1.record()
-        sync()
-        e2e_ms = e0.elapsed_time(e1) / e2e_steps
-
-    ms_per_step, e2e_ms = max_over_ranks([ms_per_step, e2e_ms], dist, device)
-
-    if rank == 0:
-        tf = lambda flop, ms: flop / (ms * 1e-3) / 1e12
-        gb = lambda byt, ms: byt / (ms * 1e-3) / 1e9
-        ms = dict(zip(STAGES, stage_ms))
-        pre_gbs, pre_tf = gb(hp.bytes_prefill, ms["prefill"]), tf(hp.flop_prefill, ms["prefill"])
-        ai = hp.flop_prefill / hp.bytes_prefill
-        bound_tf = min(peaks["bf16_tflops_sustained"], ai * peaks["hbm_gbs"] / 1e3)
-        kernels = {
-            "rope": {"ms": ms["rope"], "gbs": gb(hp.bytes_rope, ms["rope"]), "frac_hbm": gb(hp.bytes_rope, ms["rope"]) / peaks["hbm_gbs"]},
-            "prefill": {"ms": ms["prefill"], "useful_tflops": pre_tf, "gbs": pre_gbs,
-                        "frac_bf16_burst": pre_tf / peaks["bf16_tflops"],
-                        "frac_bf16_sustained": pre_tf / peaks["bf16_tflops_sustained"],
-                        "arith_intensity": ai, "binding_roofline_tflops": bound_tf, "frac_binding": pre_tf / bound_tf},
-            "path_scores": {"ms": ms["path_scores"], "gbs": gb(hp.bytes_scores, ms["path_scores"]),
-                            "frac_hbm": gb(hp.bytes_scores, ms["path_scores"]) / peaks["hbm_gbs"]},
-            "topk": {"ms": ms["topk"]},
-            "prefill_query_only": None if qo_ms is None else {
-                "ms": qo_ms, "useful_tflops": tf(hp.flop_query_only, qo_ms), "gbs": gb(hp.bytes_query_only, qo_ms),
-                "frac_hbm": gb(hp.bytes_query_only, qo_ms) / peaks["hbm_gbs"],
-                "note": "SP_ROWS_QUERY_ONLY (cached preamble/doc KV, Algorithm 3's query batch); not part of the step"},
-            "decode": {"ms": ms["decode"], "steps": hp.steps_dec, "gbs": gb(hp.bytes_decode, ms["decode"]),
-                       "frac_hbm": gb(hp.bytes_decode, ms["decode"]) / peaks["hbm_gbs"],
-                       "kernel_only_ms_per_launch": decode_kernel_ms,
-                       "kernel_only_gbs": gb(hp.bytes_decode / hp.steps_dec, decode_kernel_ms),
-                       "kernel_only_frac_hbm": gb(hp.bytes_decode / hp.steps_dec, decode_kernel_ms) / peaks["hbm_gbs"],
-                       "kv_sets": len(hp.kv_sets),
-                       "includes": "1 rope launch (q and the new key) + 1 decode launch per token" + ("" if args.no_graph else ", replayed from a CUDA graph")},
-        }
-        roof_prefill = {"kernel": "prefill_tc_kernel (sp_superpose_prefill)", "bound": "hbm", "achieved": pre_gbs,
-                        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": pre_gbs / peaks["hbm_gbs"],
-                        "traffic": NCU_TRAFFIC_BYTES.get(("prefill", cfg.name)), "peak_source": peaks["source"],
-                        "algorithmic_bytes": hp.bytes_prefill, "launch_ms": ms["prefill"], "useful_tflops": pre_tf,
-                        "frac_bf16_sustained": pre_tf / peaks["bf16_tflops_sustained"]}
-        dec_gbs = gb(hp.bytes_decode / hp.steps_dec, decode_kernel_ms)
-        roof_decode = {"kernel": "decode_kernel (sp_pruned_decode)", "bound": "hbm", "achieved": dec_gbs,
-                       "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"],
-                       "traffic": NCU_TRAFFIC_BYTES.get(("decode", cfg.name)), "peak_source": peaks["source"],
-                       "algorithmic_bytes": hp.bytes_decode / hp.steps_dec, "launch_ms": decode_kernel_ms,
-                       "launches_per_step": hp.steps_dec}
-        # the dominant kernel = the one with the largest total device time in a step
-        roofline = roof_decode if decode_kernel_ms * hp.steps_dec > ms["prefill"] else roof_prefill
+        def brief(w):
+            k = w["kernels"]
+            return {"workload": w["workload"], "ms_per_step": w["ms_per_step"], "steps": w["steps"],
+                    "value": w["value"], "tokens": w["config"]["tokens"], "allowed_pairs": w["config"]["allowed_pairs"],
+                    "useful_vs_full_causal": w["useful_vs_full_causal"], "roofline": w["roofline"],
+                    "roofline_decode": w["roofline_decode"], "kernels": k}
         line = {
-            "metric": METRIC, "value": aggregate_value(hp.flop_prefill, ms_per_step, world), "unit": UNIT,
+            "metric": METRIC, "value": aggregate_value(main["flop_prefill"], ms_per_step, world), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": cfg.dtype, "data": "synthetic",
-            "config": {"workload": cfg.name, "prompts_per_gpu": hp.B, "paths": hp.lay.n_paths,
-                       "tokens": hp.lay.total_tokens, "heads": hp.H, "head_dim": hp.D, "vocab": cfg.vocab,
-                       "top_k": cfg.top_k, "decode_steps": hp.steps_dec, "allowed_pairs": hp.pairs, "decode_kv_sets": len(hp.kv_sets),
-                       "l2": "inputs larger than L2" if flush is None else "L2 flushed between steps",
-                       "parallelism": f"dp{world} (independent prompts per GPU, no collective)"},
-            "roofline": roofline,
-            "roofline_prefill": roof_prefill,
-            "kernels": kernels,
-            "e2e": None if not e2e_steps else {
-                "value": aggregate_value(hp.flop_prefill, e2e_ms, world), "unit": UNIT, "ms_per_step": e2e_ms,
-                "steps": e2e_steps, "h2d_bytes_per_step": bi, "d2h_bytes_per_step": bo},
-            "gpu_launches": hp.launches * args.steps,
-            "clocks": clocks,
-            "input_generation_s": hp.gen_s,
+            "frac_bf16_sustained": main["frac_bf16_sustained"],
+            "config": dict(main["config"], parallelism=f"dp{world} (independent prompts per GPU, no collective)"),
+            "useful_vs_full_causal": main["useful_vs_full_causal"],
+            "roofline": main["roofline"], "roofline_decode": main["roofline_decode"], "kernels": main["kernels"],
+            "workloads": [brief(w) for w in extra],
+            "e2e": None if not main["e2e"] else {
+                "value": aggregate_value(main["flop_prefill"], e2e_ms, world), "unit": UNIT, "ms_per_step": e2e_ms,
+                "steps": main["e2e"]["steps"], "h2d_bytes_per_step": main["e2e"]["h2d"],
+                "d2h_bytes_per_step": main["e2e"]["d2h"]},
+            "gpu_launches": main["launches_per_step"] * args.steps,
+            "clocks": main["clocks"],
+            "input_generation_s": main["input_generation_s"],
         }
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(cfg, steps=1, warmup=0, budget_s=15.0)[0]
@@ -539,6 +625,17 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def launcher_command(n_gpus: int, argv):
+    """`bench.py --gpus N` started as a plain script: the command that starts N ranks of it on this
+    node (one per GPU), rendezvous on the loopback address."""
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        port = so.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -549,9 +646,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch the decode loop eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling aid)")
+    ap.add_argument("--no-extra", action="store_true", help="skip the cfg3 / cfg4 passes that follow the default workload")
     ap.add_argument("--prompts", type=int, default=None, help="override the prompts per GPU (profiling aid)")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the decode steps (profiling aid)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(subprocess.call(launcher_command(args.gpus, sys.argv[1:])))
     if args.impl == "reference":
         run_reference(args)
     else:

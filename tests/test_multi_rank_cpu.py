@@ -54,3 +54,21 @@ def test_reference_arm_runs_on_rank_zero_only():
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_gpus_flag_starts_the_ranks_itself():
+    """`bench.py --gpus 2` started as a plain script launches two ranks of itself (loopback
+    rendezvous); with the reference arm, which needs no GPU, rank 0 alone prints the line."""
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.launcher_command(2, ["--gpus", "2", "--impl", "reference"])
+    assert "--nproc-per-node=2" in cmd and "127.0.0.1" in cmd and cmd[-3:] == ["--gpus", "2", "--impl", "reference"][-3:]
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference",
+                        "--workload", "cfg0", "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True,
+                       timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                                   # rank 1 printed nothing
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2
