@@ -15,8 +15,14 @@
  *    memory is passed in as (ws, ws_bytes), sized by the *_workspace_bytes functions.
  *  - All calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL =
  *    default stream).  Arguments the host can check are checked before any launch.
- *  - Device-detected problems (a bounded wait that ran out) are recorded in the first
- *    4 bytes of the workspace and read back by sp_check_status().
+ *  - Device-detected problems (a bounded wait that ran out; a layout whose device arrays
+ *    contradict the host scalars: a segment outside [0, T), a length above max_pre_len /
+ *    max_path_len, a negative length) are recorded in the first 4 bytes of the workspace and
+ *    read back by sp_check_status().  The layout arrays live in device memory, so without a
+ *    host_mirror the host cannot see them: the kernels check them instead, skip what is
+ *    inconsistent (nothing outside the caller's tensors is read or written) and report it.
+ *    The library built with -DSP_DEBUG_BOUNDS additionally checks every pair of segments for
+ *    overlap on the device.
  *  - Tensors are dense, row-major.  Data pointers must be 16-byte aligned and
  *    n_heads * head_dim * element size must be a multiple of 16 bytes.
  *  - dtype selects storage: SP_F32 (float) or SP_BF16 (bfloat16).  Accumulation is
@@ -44,13 +50,20 @@ typedef enum {
     SP_ERR_UNSUPPORTED = 2,   /* valid but not implemented (e.g. head_dim)                */
     SP_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or too small               */
     SP_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed                      */
-    SP_ERR_TIMEOUT = 5        /* a bounded device-side wait expired (sp_check_status)     */
+    SP_ERR_TIMEOUT = 5,       /* a bounded device-side wait expired (sp_check_status)     */
+    SP_ERR_LAYOUT = 6         /* the device-resident layout arrays are inconsistent
+                                 (sp_check_status; the affected segments were skipped)    */
 } sp_status;
 
 enum { SP_F32 = 0, SP_BF16 = 1 };
 enum { SP_ROWS_ALL = 0, SP_ROWS_QUERY_ONLY = 1 };
 enum { SP_POS_EQUILIBRIUM = 0, SP_POS_LEFT_ALIGNED = 1 };
 enum { SP_ROPE_HALF_SPLIT = 0, SP_ROPE_INTERLEAVED = 1 };
+
+/* HOST copies of the six index arrays of an sp_layout (same lengths and meaning). */
+typedef struct {
+    const int32_t *prompt_path_off, *pre_start, *pre_len, *path_start, *doc_len, *qry_len;
+} sp_layout_host;
 
 typedef struct {
     int32_t n_prompts;               /* B                                                  */
@@ -64,6 +77,11 @@ typedef struct {
     int64_t total_tokens;            /* T: number of packed rows of Q / K / V / out        */
     int32_t max_pre_len;             /* >= every pre_len[b]            (host scalar)       */
     int32_t max_path_len;            /* >= every doc_len[i]+qry_len[i] (host scalar)       */
+    const sp_layout_host *host_mirror; /* HOST, nullable: when given, every call validates the
+                                        whole layout on the host before launching (offsets
+                                        ascending, lengths >= 0 and within the two maxima, every
+                                        segment inside [0, T), no two segments overlapping) and
+                                        returns SP_ERR_INVALID_ARG on a violation              */
 } sp_layout;
 
 /* Message for the calling thread's last failing call ("" if none).  HOST. */
@@ -273,7 +291,10 @@ int sp_pruned_decode_static(const void *q, const void *k_cache, const void *v_ca
 /*
  * Reads the device status word at the start of a workspace after synchronising `stream`.
  * Returns SP_OK, SP_ERR_TIMEOUT (a bounded wait expired; the outputs of that call are
- * not valid) or SP_ERR_CUDA.  The word is cleared by the next call that uses the workspace.
+ * not valid), SP_ERR_LAYOUT (the layout arrays on the device were inconsistent; what could not
+ * be trusted was skipped, so the outputs are incomplete) or SP_ERR_CUDA.  The word is cleared
+ * by the next sp_superpose_prefill / sp_pruned_decode call that uses the workspace;
+ * sp_path_scores has nothing to report and leaves the word alone.
  */
 int sp_check_status(const void *ws, void *stream);
 

@@ -14,10 +14,11 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsp_b200.so")
+# SP_B200_DEBUG_BOUNDS=1 selects the twin built with -DSP_DEBUG_BOUNDS (extra device-side layout checks)
+LIB_PATH = os.path.join(_HERE, "libsp_b200_debug.so" if os.environ.get("SP_B200_DEBUG_BOUNDS") == "1" else "libsp_b200.so")
 
 SP_OK = 0
-SP_ERR_INVALID_ARG, SP_ERR_UNSUPPORTED, SP_ERR_WORKSPACE, SP_ERR_CUDA, SP_ERR_TIMEOUT = 1, 2, 3, 4, 5
+SP_ERR_INVALID_ARG, SP_ERR_UNSUPPORTED, SP_ERR_WORKSPACE, SP_ERR_CUDA, SP_ERR_TIMEOUT, SP_ERR_LAYOUT = 1, 2, 3, 4, 5, 6
 SP_F32, SP_BF16 = 0, 1
 SP_ROWS_ALL, SP_ROWS_QUERY_ONLY = 0, 1
 SP_POS_EQUILIBRIUM, SP_POS_LEFT_ALIGNED = 0, 1
@@ -39,6 +40,10 @@ class SpError(RuntimeError):
         self.code = code
 
 
+class _CLayoutHost(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("prompt_path_off", "pre_start", "pre_len", "path_start", "doc_len", "qry_len")]
+
+
 class _CLayout(ctypes.Structure):
     _fields_ = [
         ("n_prompts", ctypes.c_int32), ("n_paths", ctypes.c_int32),
@@ -47,6 +52,7 @@ class _CLayout(ctypes.Structure):
         ("doc_len", ctypes.c_void_p), ("qry_len", ctypes.c_void_p),
         ("total_tokens", ctypes.c_int64),
         ("max_pre_len", ctypes.c_int32), ("max_path_len", ctypes.c_int32),
+        ("host_mirror", ctypes.POINTER(_CLayoutHost)),
     ]
 
 
@@ -138,14 +144,17 @@ class DeviceLayout:
         return self.arrays[0]
 
     @staticmethod
-    def from_host(lay, device="cuda") -> "DeviceLayout":
-        def dev(a):
-            return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
-        arrs = tuple(dev(a) for a in (lay.prompt_path_off, lay.pre_start, lay.pre_len,
-                                      lay.path_start, lay.doc_len, lay.qry_len))
+    def from_host(lay, device="cuda", mirror: bool = True) -> "DeviceLayout":
+        """mirror: also hand the host copies of the index arrays to the library, which then
+        validates the whole layout on the host in every call."""
+        host = tuple(np.ascontiguousarray(a, dtype=np.int32) for a in (lay.prompt_path_off, lay.pre_start, lay.pre_len,
+                                                                       lay.path_start, lay.doc_len, lay.qry_len))
+        arrs = tuple(torch.from_numpy(a).to(device) for a in host)
+        hm = _CLayoutHost(*[a.ctypes.data for a in host]) if mirror else None
         c = _CLayout(lay.n_prompts, lay.n_paths, *[a.data_ptr() for a in arrs],
-                     lay.total_tokens, lay.max_pre_len, lay.max_path_len)
-        return DeviceLayout(c, arrs, lay.n_prompts, lay.n_paths, lay.total_tokens,
+                     lay.total_tokens, lay.max_pre_len, lay.max_path_len,
+                     ctypes.pointer(hm) if mirror else None)
+        return DeviceLayout(c, arrs + host + (hm,), lay.n_prompts, lay.n_paths, lay.total_tokens,
                             lay.max_pre_len, lay.max_path_len)
 
 

@@ -1,4 +1,5 @@
-"""Builds the CUDA library in-tree: every csrc/*.cu -> libsp_b200.so (sm_100a only)."""
+"""Builds the CUDA library in-tree: every csrc/*.cu -> libsp_b200.so (sm_100a only), and the same
+sources with -DSP_DEBUG_BOUNDS (extra device-side layout checks) -> libsp_b200_debug.so."""
 from __future__ import annotations
 
 import os
@@ -10,6 +11,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libsp_b200.so")
+OBJ_DEBUG = os.path.join(HERE, "_build_debug")
+LIB_DEBUG = os.path.join(HERE, "libsp_b200_debug.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -27,12 +30,12 @@ def _deps_mtime():
     return max(os.path.getmtime(h) for h in hdrs)
 
 
-def _compile(src: str, verbose: bool) -> str:
-    obj = os.path.join(OBJ, src[:-3] + ".o")
+def _compile(src: str, verbose: bool, obj_dir: str = OBJ, extra=()) -> str:
+    obj = os.path.join(obj_dir, src[:-3] + ".o")
     path = os.path.join(CSRC, src)
     if os.path.exists(obj) and os.path.getmtime(obj) >= max(os.path.getmtime(path), _deps_mtime()):
         return obj
-    cmd = ["nvcc", *NVCC_FLAGS, "-c", path, "-o", obj]
+    cmd = ["nvcc", *NVCC_FLAGS, *extra, "-c", path, "-o", obj]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or res.returncode:
         sys.stderr.write(f"$ {' '.join(cmd)}\n{res.stdout}{res.stderr}")
@@ -41,19 +44,27 @@ def _compile(src: str, verbose: bool) -> str:
     return obj
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    os.makedirs(OBJ, exist_ok=True)
+def _build_one(lib: str, obj_dir: str, extra, force: bool, verbose: bool) -> str:
+    os.makedirs(obj_dir, exist_ok=True)
     if force:
-        for f in os.listdir(OBJ):
-            os.remove(os.path.join(OBJ, f))
+        for f in os.listdir(obj_dir):
+            os.remove(os.path.join(obj_dir, f))
     with ThreadPoolExecutor(max_workers=8) as ex:
-        objs = list(ex.map(lambda s: _compile(s, verbose), _sources()))
-    if force or not os.path.exists(LIB) or os.path.getmtime(LIB) < max(os.path.getmtime(o) for o in objs):
-        tmp = LIB + f".tmp{os.getpid()}"
+        objs = list(ex.map(lambda s: _compile(s, verbose, obj_dir, extra), _sources()))
+    if force or not os.path.exists(lib) or os.path.getmtime(lib) < max(os.path.getmtime(o) for o in objs):
+        tmp = lib + f".tmp{os.getpid()}"
         subprocess.check_call(["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp, *objs,
                                "-Xcompiler", "-fPIC"])
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
+    return lib
+
+
+def build(force: bool = False, verbose: bool = False, debug: bool = True) -> str:
+    """Builds the library and (debug=True) its bounds-checking twin; returns the library's path."""
+    lib = _build_one(LIB, OBJ, (), force, verbose)
+    if debug:
+        _build_one(LIB_DEBUG, OBJ_DEBUG, ("-DSP_DEBUG_BOUNDS",), force, verbose)
+    return lib
 
 
 if __name__ == "__main__":

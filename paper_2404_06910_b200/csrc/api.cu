@@ -1,6 +1,8 @@
 // Host-side pieces of the C ABI that launch nothing: error strings, layout checks,
 // token position assignment, the device status read-back.
 #include <cstring>
+#include <utility>
+#include <vector>
 
 #include "common.cuh"
 
@@ -52,6 +54,39 @@ int check_layout(const sp_layout *lay)
     if (lay->n_paths > 0)
         SP_REQUIRE(lay->path_start && lay->doc_len && lay->qry_len, SP_ERR_INVALID_ARG,
                    "layout: per-path arrays are NULL");
+    if (lay->host_mirror == nullptr) return SP_OK;
+
+    // full validation on the caller's host copy of the arrays
+    const sp_layout_host &m = *lay->host_mirror;
+    const int B = lay->n_prompts, NP = lay->n_paths;
+    const int64_t T = lay->total_tokens;
+    if (B > 0) SP_REQUIRE(m.prompt_path_off && m.pre_start && m.pre_len, SP_ERR_INVALID_ARG, "layout: host mirror of the per-prompt arrays is NULL");
+    if (NP > 0) SP_REQUIRE(m.path_start && m.doc_len && m.qry_len, SP_ERR_INVALID_ARG, "layout: host mirror of the per-path arrays is NULL");
+    if (B > 0) SP_REQUIRE(m.prompt_path_off[0] == 0 && m.prompt_path_off[B] == NP, SP_ERR_INVALID_ARG,
+                          "layout: prompt_path_off must run from 0 to n_paths");
+    std::vector<std::pair<int64_t, int64_t>> seg;          // (first row, one past the last row)
+    seg.reserve((size_t)B + NP);
+    for (int b = 0; b < B; ++b) {
+        SP_REQUIRE(m.prompt_path_off[b] <= m.prompt_path_off[b + 1], SP_ERR_INVALID_ARG, "layout: prompt_path_off decreases at prompt %d", b);
+        SP_REQUIRE(m.pre_len[b] >= 0 && m.pre_len[b] <= lay->max_pre_len, SP_ERR_INVALID_ARG,
+                   "layout: pre_len[%d] = %d outside [0, max_pre_len = %d]", b, m.pre_len[b], lay->max_pre_len);
+        SP_REQUIRE(m.pre_start[b] >= 0 && (int64_t)m.pre_start[b] + m.pre_len[b] <= T, SP_ERR_INVALID_ARG,
+                   "layout: preamble of prompt %d leaves [0, total_tokens)", b);
+        if (m.pre_len[b]) seg.emplace_back(m.pre_start[b], (int64_t)m.pre_start[b] + m.pre_len[b]);
+    }
+    for (int i = 0; i < NP; ++i) {
+        SP_REQUIRE(m.doc_len[i] >= 0 && m.qry_len[i] >= 0 && (int64_t)m.doc_len[i] + m.qry_len[i] <= lay->max_path_len,
+                   SP_ERR_INVALID_ARG, "layout: path %d has lengths (%d, %d) outside [0, max_path_len = %d]", i, m.doc_len[i],
+                   m.qry_len[i], lay->max_path_len);
+        const int64_t n = (int64_t)m.doc_len[i] + m.qry_len[i];
+        SP_REQUIRE(m.path_start[i] >= 0 && m.path_start[i] + n <= T, SP_ERR_INVALID_ARG,
+                   "layout: path %d leaves [0, total_tokens)", i);
+        if (n) seg.emplace_back(m.path_start[i], m.path_start[i] + n);
+    }
+    std::sort(seg.begin(), seg.end());
+    for (size_t i = 1; i < seg.size(); ++i)
+        SP_REQUIRE(seg[i].first >= seg[i - 1].second, SP_ERR_INVALID_ARG,
+                   "layout: the segments starting at rows %lld and %lld overlap", (long long)seg[i - 1].first, (long long)seg[i].first);
     return SP_OK;
 }
 
@@ -115,6 +150,9 @@ int sp_check_status(const void *ws, void *stream)
     if (word == sp::STATUS_OK) return SP_OK;
     if (word == sp::STATUS_TIMEOUT)
         return sp::fail(SP_ERR_TIMEOUT, "a bounded device-side wait expired; outputs are not valid");
+    if (word == sp::STATUS_BAD_LAYOUT)
+        return sp::fail(SP_ERR_LAYOUT, "the layout arrays on the device are inconsistent with total_tokens / max_pre_len / "
+                                       "max_path_len (or overlap); the affected segments were skipped");
     return sp::fail(SP_ERR_CUDA, "unknown device status word %u", word);
 }
 

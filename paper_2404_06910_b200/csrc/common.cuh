@@ -39,7 +39,7 @@ __host__ __device__ constexpr size_t round_up(size_t x, size_t a) { return (x + 
 int check_layout(const sp_layout *lay);     // host-visible fields only (api.cu)
 
 // Device status word codes (first 4 bytes of a workspace).
-enum : uint32_t { STATUS_OK = 0, STATUS_TIMEOUT = 1 };
+enum : uint32_t { STATUS_OK = 0, STATUS_TIMEOUT = 1, STATUS_BAD_LAYOUT = 2 };
 
 int num_sms();                              // multiprocessors of the current device (api.cu)
 

@@ -35,6 +35,7 @@ struct DecodeArgs {
     float *partial;          // [B*H][n_splits][D+2]
     unsigned int *counters;  // [B*H], zero on entry
     int k, tail_cap, n_heads, n_kv_heads, n_splits;
+    int64_t total_tokens;    // T: cache segments outside [0, T) are skipped (cluster kernel)
     float scale_log2e;
     // ALiBi variant only: positions of the query token [B], of the cache rows [T] and of the
     // tail rows [B, tail_cap], and the per-head slopes [H]
@@ -344,6 +345,8 @@ decode_cluster_kernel(const __grid_constant__ DecodeArgs a, const __grid_constan
                 row = (int64_t)b * a.tail_cap;
             }
         }
+        // a cache segment that the device-side layout puts outside the tensors is not read at all
+        if (sgm <= a.k && (len < 0 || row < 0 || row + len > a.total_tokens)) { len = 0; row = 0; }
         seg_k[sgm] = kc + row * row_elems;
         seg_v[sgm] = vc + row * row_elems;
         if (ALIBI) seg_pos[sgm] = (sgm == a.k + 1 && len ? a.tail_pos : a.cache_pos) + row;
@@ -724,7 +727,7 @@ static int decode_with_workspace(const void *q, const void *k_cache, const void 
     a.kept_idx = kept_idx; a.tail_len = tail_len; a.out = out; a.lse = lse;
     a.counters = nullptr; a.partial = nullptr;
     a.k = k; a.tail_cap = tail_cap; a.n_heads = n_heads; a.n_kv_heads = n_kv_heads;
-    a.n_splits = 1; a.scale_log2e = scale * kLog2eD;
+    a.n_splits = 1; a.scale_log2e = scale * kLog2eD; a.total_tokens = lay->total_tokens;
     a.q_pos = q_pos; a.cache_pos = cache_pos; a.tail_pos = tail_pos; a.slopes = slopes;
 
     DecodeRope rope = {};
@@ -873,7 +876,7 @@ extern "C" int sp_pruned_decode_static(const void *q, const void *k_cache, const
     a.counters = reinterpret_cast<unsigned int *>(scratch);
     a.partial = reinterpret_cast<float *>(scratch + cbytes);
     a.k = k; a.tail_cap = tail_cap; a.n_heads = n_heads; a.n_kv_heads = n_kv_heads;
-    a.n_splits = n_splits; a.scale_log2e = scale * kLog2eD;
+    a.n_splits = n_splits; a.scale_log2e = scale * kLog2eD; a.total_tokens = lay->total_tokens;
     a.q_pos = nullptr; a.cache_pos = nullptr; a.tail_pos = nullptr; a.slopes = nullptr;
 
     if (dtype == SP_BF16)

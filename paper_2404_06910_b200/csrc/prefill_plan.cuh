@@ -25,9 +25,17 @@ struct PlanArgs {
     const int32_t *ppo, *pre_start, *pre_len, *path_start, *doc_len, *qry_len;
     int n_prompts, n_paths, rows_mode;
     int tile_rows;                    // query rows per tile
+    int max_pre_len, max_path_len;    // the host's bounds on the lengths (they sized the tile list)
+    int64_t total_tokens;             // T: every segment must lie inside [0, T)
+    int64_t max_tiles;                // capacity of the tile list
     TcHeader *hdr;
     TcTile *tiles;
 };
+
+// What the host cannot check, the plan kernel does: a segment whose device-side numbers
+// contradict the host scalars (negative or oversized length, rows outside [0, T)) gets no tiles
+// and the status word reports it, so nothing outside the caller's tensors is ever touched and
+// the tile list cannot outgrow the workspace that was sized from those scalars.
 
 static __global__ void __launch_bounds__(1024) prefill_plan_kernel(const PlanArgs a)
 {
@@ -40,8 +48,11 @@ static __global__ void __launch_bounds__(1024) prefill_plan_kernel(const PlanArg
     for (int base = 0; base < n_seq; base += 1024) {
         const int s = base + threadIdx.x;
         int first = 0, rows = 0, own_row = 0, pre_row = 0, pre_n = 0;
+        bool bad = false;
         if (s < a.n_prompts) {
-            if (a.rows_mode == SP_ROWS_ALL) { rows = a.pre_len[s]; own_row = a.pre_start[s]; }
+            const int len = a.pre_len[s], row = a.pre_start[s];
+            bad = len < 0 || len > a.max_pre_len || row < 0 || (int64_t)row + len > a.total_tokens;
+            if (a.rows_mode == SP_ROWS_ALL && !bad) { rows = len; own_row = row; }
         } else if (s < n_seq) {
             const int i = s - a.n_prompts;
             int lo = 0, hi = a.n_prompts - 1;
@@ -51,9 +62,23 @@ static __global__ void __launch_bounds__(1024) prefill_plan_kernel(const PlanArg
             }
             pre_row = a.pre_start[lo]; pre_n = a.pre_len[lo];
             own_row = a.path_start[i];
-            first = a.rows_mode == SP_ROWS_QUERY_ONLY ? a.doc_len[i] : 0;
-            rows = a.doc_len[i] + a.qry_len[i] - first;
+            const int dl = a.doc_len[i], ql = a.qry_len[i];
+            bad = dl < 0 || ql < 0 || (int64_t)dl + ql > a.max_path_len || own_row < 0 ||
+                  (int64_t)own_row + dl + ql > a.total_tokens ||
+                  pre_n < 0 || pre_n > a.max_pre_len || pre_row < 0 || (int64_t)pre_row + pre_n > a.total_tokens;
+#ifdef SP_DEBUG_BOUNDS
+            // debug build: no other segment may share a row with this path (every pair is looked at)
+            for (int o = 0; o < n_seq && !bad; ++o) {
+                if (o == s) continue;
+                const int orow = o < a.n_prompts ? a.pre_start[o] : a.path_start[o - a.n_prompts];
+                const int olen = o < a.n_prompts ? a.pre_len[o] : a.doc_len[o - a.n_prompts] + a.qry_len[o - a.n_prompts];
+                bad = olen > 0 && dl + ql > 0 && orow < own_row + dl + ql && own_row < orow + olen;
+            }
+#endif
+            first = a.rows_mode == SP_ROWS_QUERY_ONLY ? dl : 0;
+            rows = bad ? 0 : dl + ql - first;
         }
+        if (bad) a.hdr->status = STATUS_BAD_LAYOUT;
         const int nt = (rows + a.tile_rows - 1) / a.tile_rows;
         int incl = nt;
 #pragma unroll
@@ -66,7 +91,7 @@ static __global__ void __launch_bounds__(1024) prefill_plan_kernel(const PlanArg
         int before = running;
         for (int w = 0; w < warp; ++w) before += warp_tot[w];
         int off = before + incl - nt;
-        for (int t = 0; t < nt; ++t) {
+        for (int t = 0; t < nt && off + t < a.max_tiles; ++t) {
             TcTile tl;
             tl.q_off = first + t * a.tile_rows;
             tl.q_row = own_row + tl.q_off;
@@ -79,7 +104,7 @@ static __global__ void __launch_bounds__(1024) prefill_plan_kernel(const PlanArg
         if (threadIdx.x == 1023) running = before + incl;
         __syncthreads();
     }
-    if (threadIdx.x == 0) a.hdr->n_tiles = (uint32_t)running;
+    if (threadIdx.x == 0) a.hdr->n_tiles = (uint32_t)min((int64_t)running, a.max_tiles);
 }
 
 static inline int64_t plan_max_tiles(int n_prompts, int n_paths, int max_pre_len, int max_path_len, int tile_rows)

@@ -346,6 +346,8 @@ int launch_prefill_qonly(const void *q, const void *k, const void *v, const sp_l
     pa.ppo = lay->prompt_path_off; pa.pre_start = lay->pre_start; pa.pre_len = lay->pre_len;
     pa.path_start = lay->path_start; pa.doc_len = lay->doc_len; pa.qry_len = lay->qry_len;
     pa.n_prompts = lay->n_prompts; pa.n_paths = lay->n_paths; pa.rows_mode = SP_ROWS_QUERY_ONLY; pa.tile_rows = kQM;
+    pa.max_pre_len = lay->max_pre_len; pa.max_path_len = lay->max_path_len; pa.total_tokens = lay->total_tokens;
+    pa.max_tiles = plan_max_tiles(lay->n_prompts, lay->n_paths, lay->max_pre_len, lay->max_path_len, kQM);
     pa.hdr = hdr; pa.tiles = tiles;
     prefill_plan_kernel<<<1, 1024, 0, st>>>(pa);
     SP_CUDA(cudaGetLastError());

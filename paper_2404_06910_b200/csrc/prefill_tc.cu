@@ -17,8 +17,6 @@
 // share an SM (256 TMEM columns each).  A small plan kernel turns the ragged layout into a
 // tile list.  Every mbarrier wait is bounded: on expiry the block records a timeout in the
 // workspace status word, unwinds, frees its TMEM and exits.
-#include <cstdlib>
-
 #include "common.cuh"
 #include "prefill_plan.cuh"
 #include "tc_ptx.cuh"
@@ -534,6 +532,12 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
 }
 
 // ---- host side ---------------------------------------------------------------------------
+// Failure-detection test hook (host-injected, no GPU fault): while set, the producer loads no
+// tile, every bounded wait expires, the blocks unwind and the call reports SP_ERR_TIMEOUT
+// through the workspace status word.  Set only through sp_test_stall_producer(), a symbol for
+// the test suite that the public header does not declare.
+static bool g_stall_producer = false;
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -596,6 +600,8 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
     pa.ppo = lay->prompt_path_off; pa.pre_start = lay->pre_start; pa.pre_len = lay->pre_len;
     pa.path_start = lay->path_start; pa.doc_len = lay->doc_len; pa.qry_len = lay->qry_len;
     pa.n_prompts = lay->n_prompts; pa.n_paths = lay->n_paths; pa.rows_mode = rows; pa.tile_rows = kBM;
+    pa.max_pre_len = lay->max_pre_len; pa.max_path_len = lay->max_path_len; pa.total_tokens = lay->total_tokens;
+    pa.max_tiles = plan_max_tiles(lay->n_prompts, lay->n_paths, lay->max_pre_len, lay->max_path_len, kBM);
     pa.hdr = hdr; pa.tiles = tiles;
     prefill_plan_kernel<<<1, 1024, 0, st>>>(pa);
     SP_CUDA(cudaGetLastError());
@@ -605,11 +611,7 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
     p.n_heads = n_heads; p.kv_group = n_heads / n_kv_heads;
     p.total_tokens = lay->total_tokens; p.scale_log2e = scale * kLog2eT;
     p.pos = pos; p.slopes = slopes;
-    // Failure-detection test hook (host-injected, no GPU fault): with SP_TEST_STALL_PRODUCER=1 in
-    // the environment no tile is ever loaded, every bounded wait expires, the blocks unwind and
-    // the call reports SP_ERR_TIMEOUT through the workspace status word.
-    const char *stall = std::getenv("SP_TEST_STALL_PRODUCER");
-    p.stall_producer = (stall && stall[0] == '1') ? 1 : 0;
+    p.stall_producer = g_stall_producer ? 1 : 0;      // test hook, see sp_test_stall_producer below
 
     const int64_t items = max_tiles(lay->n_prompts, lay->n_paths, lay->max_pre_len, lay->max_path_len) * n_heads;
     if (items == 0) return SP_OK;
@@ -627,3 +629,5 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
 }
 
 }  // namespace sp
+
+extern "C" void sp_test_stall_producer(int on) { sp::g_stall_producer = on != 0; }

@@ -1,5 +1,5 @@
 """Failure detection without a GPU fault: the producer of the tensor-core prefill is told (on
-the host) to load nothing, so every device-side wait runs into its limit.  The kernel must
+the host, through a test-only symbol) to load nothing, so every device-side wait runs into its limit.  The kernel must
 unwind by itself, report SP_ERR_TIMEOUT through the workspace status word, and leave the
 context usable: the next ordinary call gives the same result as before."""
 import math
@@ -15,7 +15,7 @@ from workloads import build_layout
 pytestmark = pytest.mark.gpu
 
 
-def test_prefill_bounded_waits_report_timeout_and_context_survives(monkeypatch):
+def test_prefill_bounded_waits_report_timeout_and_context_survives():
     lay = build_layout([32], [[100, 40]], [[24, 24]])
     H, D = 2, 128
     g = torch.Generator().manual_seed(5)
@@ -32,12 +32,14 @@ def test_prefill_bounded_waits_report_timeout_and_context_survives(monkeypatch):
     good = run()
     sp.sp_check_status(ws)
 
-    monkeypatch.setenv("SP_TEST_STALL_PRODUCER", "1")
-    run()
-    with pytest.raises(sp.SpError) as e:
-        sp.sp_check_status(ws)
-    assert e.value.code == sp.SP_ERR_TIMEOUT
-    monkeypatch.delenv("SP_TEST_STALL_PRODUCER")
+    sp.lib.sp_test_stall_producer(1)            # test-only symbol: the producer loads nothing from now on
+    try:
+        run()
+        with pytest.raises(sp.SpError) as e:
+            sp.sp_check_status(ws)
+        assert e.value.code == sp.SP_ERR_TIMEOUT
+    finally:
+        sp.lib.sp_test_stall_producer(0)
 
     again = run()
     sp.sp_check_status(ws)                      # status word is cleared by the next call

@@ -423,6 +423,43 @@ def test_topk_ties_nan_and_short_prompts():
         oracle.prune_topk(s, ppo, 0)
 
 
+def test_topk_posterior_when_no_score_is_finite():
+    """Cases the paper is silent on, expected values written out by hand from the reading taken
+    (NaN ranks below every number and counts as -inf; equal scores keep the lower id first; the
+    posterior of a prompt with no score above -inf is zero everywhere, not NaN)."""
+    ninf, nan = -np.inf, np.nan
+    idx, post = oracle.prune_topk(np.array([ninf, nan, ninf], np.float32), np.array([0, 3], np.int32), 3)
+    assert idx.tolist() == [[0, 2, 1]] and post.tolist() == [[0.0, 0.0, 0.0]]
+    idx, post = oracle.prune_topk(np.array([nan, nan], np.float32), np.array([0, 2], np.int32), 1)
+    assert idx.tolist() == [[0]] and post.tolist() == [[0.0]]
+    # one finite score among -inf and NaN takes the whole posterior
+    idx, post = oracle.prune_topk(np.array([ninf, 3.0, ninf, nan], np.float32), np.array([0, 4], np.int32), 2)
+    assert idx.tolist() == [[1, 0]] and post.tolist() == [[1.0, 0.0]]
+    # two prompts side by side: the degenerate one does not disturb its neighbour
+    idx, post = oracle.prune_topk(np.array([ninf, ninf, 0.0, 0.0], np.float32), np.array([0, 2, 4], np.int32), 2)
+    assert idx.tolist() == [[0, 1], [2, 3]] and post.tolist() == [[0.0, 0.0], [0.5, 0.5]]
+
+
+def test_positions_with_empty_documents_and_empty_preamble():
+    """Eq. 1 with a zero-length document (it has no term in the harmonic mean and no rows of its
+    own; its query copy still starts at P + S like every other) and with no preamble
+    (max of the empty set + 1 = 0).  Expected values derived by hand:
+    L = {0, 2, 4}: S = 2 / (1/2 + 1/4) = 8/3, steps 4/3 and 2/3, queries at 2 + 8/3 = 14/3."""
+    pos, S, nxt = oracle.positions(2, [0, 2, 4], 1)
+    want = [0, 1,                      # preamble
+            14 / 3,                    # empty document: only its query copy
+            2, 10 / 3, 14 / 3,         # document of 2 (step 4/3), query
+            2, 8 / 3, 10 / 3, 4, 14 / 3]
+    np.testing.assert_allclose(pos, want, rtol=0, atol=1e-12)
+    assert S == pytest.approx(8 / 3, abs=1e-12) and nxt == pytest.approx(17 / 3, abs=1e-12)
+    pos, S, nxt = oracle.positions(0, [2, 4], 1)
+    np.testing.assert_allclose(pos, [0, 4 / 3, 8 / 3, 0, 2 / 3, 4 / 3, 2, 8 / 3], rtol=0, atol=1e-12)
+    assert nxt == pytest.approx(11 / 3, abs=1e-12)
+    # every document empty: S = 0, the queries follow the preamble directly
+    pos, S, nxt = oracle.positions(3, [0, 0], 2)
+    assert pos.tolist() == [0, 1, 2, 3, 4, 3, 4] and S == 0.0 and nxt == 5.0
+
+
 # ---------------------------------------------------------------- O6 decode
 def _decode_setup():
     lay = build_layout([3, 2], [[4, 2, 5], [3, 6]], [[2, 2, 2], [3, 3]])

@@ -5,14 +5,16 @@ inference server whose pool is already carved up, a plugin that may not touch th
 allocator).  For them the library carries its own fixed split-KV scratch array.  This test
 drives that entry point through the C ABI twice in a row -- the second call finds the
 first call's leftovers in the shared array -- and checks both results against the ordinary
-entry point that takes a caller workspace.  It is collected last on purpose, and it passes
-on its own in a fresh process as well as after the other GPU tests."""
+entry point that takes a caller workspace and against the CPU oracle, and that the device's
+free memory is the same before and after the call.  It is collected last on purpose, and it
+passes on its own in a fresh process as well as after the other GPU tests."""
 import math
 
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2404_06910_b200 as sp
 from helpers import dev, f32, rel_l2, workspace
 from workloads import build_layout
@@ -50,11 +52,19 @@ def test_static_scratch_decode_matches_workspace_decode_twice(dtype, tol):
                             ref, ref_lse, ws)
         got = torch.full_like(ref, float("nan"))
         got_lse = torch.full_like(ref_lse, float("nan"))
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         sp.sp_pruned_decode_static(d["q"], d["kc"], d["vc"], dl, d["kept"], 2, d["tk"], d["tv"], d["tail_len"], 6,
                                    scale, got, got_lse)
         torch.cuda.synchronize()
+        if call == 1:       # (the very first call may load the kernel's code; the second one must take nothing)
+            assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
         assert not torch.isnan(got).any(), f"call {call}: rows left unwritten"
         assert rel_l2(f32(got), f32(ref)) <= tol, f"call {call}"
+        want, want_lse = oracle.pruned_decode(f32(x["q"]), f32(x["kc"]), f32(x["vc"]), lay, x["kept"], f32(x["tk"]),
+                                              f32(x["tv"]), x["tail_len"], scale)
+        assert rel_l2(f32(got), want) <= tol, f"call {call}: against the oracle"
+        np.testing.assert_allclose(got_lse.cpu().numpy(), want_lse, atol=1e-5 if dtype == torch.float32 else 2e-2)
         np.testing.assert_allclose(got_lse.cpu().numpy(), ref_lse.cpu().numpy(), atol=1e-5 if dtype == torch.float32 else 2e-2)
 
 
