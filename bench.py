@@ -400,10 +400,11 @@ def measure_workload(cfg, sp, device, args, rank, dist, peaks, steps, warmup, wi
     # decode kernel alone (no rotation of the new rows), replayed from a graph: the per-launch
     # figure of that kernel; cold = KV sets rotate (as in the step), warm = one set re-read
     n_dec = hp.steps_dec
-    dec_cold_ms = timed(graph_of(lambda: hp.decode_loop(with_rope=False)).replay, per=n_dec)
+    plain_loop = lambda: hp.decode_loop(with_rope=False)
+    dec_cold_ms = timed(plain_loop if args.no_graph else graph_of(plain_loop).replay, per=n_dec)
     sets = hp.kv_sets
     hp.kv_sets = sets[:1]
-    dec_warm_ms = timed(graph_of(lambda: hp.decode_loop(with_rope=False)).replay, per=n_dec)
+    dec_warm_ms = timed(plain_loop if args.no_graph else graph_of(plain_loop).replay, per=n_dec)
     hp.kv_sets = sets
     # the decode step as an application without CUDA graphs would issue it: eager launches
     dec_eager_ms = timed(lambda: hp.decode_loop(), reps=3, per=n_dec)
@@ -554,6 +555,90 @@ def run_ours(args):
 
 
 # ---------------------------------------------------------------------------------------
+def run_widened(args):
+    """Timings of the rows beyond the first path (not part of the step, printed as one JSON line):
+    the ALiBi variants of the prefill and the decode on the chosen workload, and an iterative
+    superposition workload (Section 4.3: t rounds, the k documents kept in a round join the
+    shared prefix of the next) with document lengths around the paper's multi-hop setting
+    (Appendix D: 20 documents, about 121 tokens each)."""
+    import paper_2404_06910_b200 as sp
+    from workloads import build_layout, next_round_layout
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    hbm = peaks["hbm_gbs"]
+    cfg = get_config(args.workload)
+    hp = HotPath(cfg, cfg.seed, sp, device, args.prompts, args.decode_steps)
+    H, D, B = hp.H, hp.D, hp.B
+
+    def timed(fn, reps=7, per=1):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) / per)
+        return float(np.median(ts))
+
+    gb = lambda byt, ms: byt / (ms * 1e-3) / 1e9
+    slopes = torch.tensor([2.0 ** (-8.0 * (h + 1) / H) for h in range(H)], dtype=torch.float32, device=device)
+    plain_ms = timed(lambda: sp.sp_superpose_prefill(hp.q, hp.k, hp.v, hp.dl, hp.scale, hp.out, None, hp.ws_pre))
+    alibi_ms = timed(lambda: sp.sp_superpose_prefill_alibi(hp.q, hp.k, hp.v, hp.dl, hp.pos, slopes, hp.scale, hp.out,
+                                                           None, hp.ws_pre))
+    hp.step()
+    torch.cuda.synchronize()
+    hp.bytes_decode = hp.decode_bytes()
+    n_dec = hp.steps_dec
+    tail_pos = hp.tpos.t().contiguous()                                # [B, steps]
+    def dec_plain():
+        for t in range(n_dec):
+            sp.sp_pruned_decode(hp.dq[t], hp.k, hp.v, hp.dl, hp.kept, cfg.top_k, hp.tk, hp.tv, hp.tail_len[t], n_dec,
+                                hp.scale, hp.dec_out[t], None, hp.ws_dec)
+    def dec_alibi():
+        for t in range(n_dec):
+            sp.sp_pruned_decode_alibi(hp.dq[t], hp.k, hp.v, hp.dl, hp.kept, cfg.top_k, hp.tk, hp.tv, hp.tail_len[t],
+                                      n_dec, hp.tpos[t], hp.pos, tail_pos, slopes, hp.scale, hp.dec_out[t], None, hp.ws_dec)
+    dplain_ms, dalibi_ms = timed(dec_plain, reps=3, per=n_dec), timed(dec_alibi, reps=3, per=n_dec)
+    alibi = {"workload": cfg.name,
+             "prefill_ms": plain_ms, "prefill_alibi_ms": alibi_ms, "prefill_alibi_frac_hbm": gb(hp.bytes_prefill, alibi_ms) / hbm,
+             "decode_us": dplain_ms * 1e3, "decode_alibi_us": dalibi_ms * 1e3,
+             "decode_alibi_frac_hbm": gb(hp.bytes_decode / n_dec, dalibi_ms) / hbm,
+             "note": "decode launches issued eagerly, one KV set"}
+    del hp
+    torch.cuda.empty_cache()
+
+    # iterative superposition: lengths ~ U{60..180} (mean 120), 20 documents, preamble 32, query 24
+    rng = np.random.default_rng(20240410 + 77)
+    n_prompts, n_docs, k_keep, rounds = 64, 20, 2, 3
+    lay = build_layout([32] * n_prompts, [rng.integers(60, 181, size=n_docs) for _ in range(n_prompts)],
+                       [[24] * n_docs] * n_prompts)
+    iters = []
+    for r in range(rounds):
+        T = lay.total_tokens
+        g = torch.Generator(device=device); g.manual_seed(100 + r)
+        q, k, v = (torch.randn(T, H, D, device=device, generator=g).mul_(D ** -0.5).bfloat16() for _ in range(3))
+        out = torch.empty_like(q)
+        dl = sp.DeviceLayout.from_host(lay, device)
+        ws = torch.zeros(max(256, sp.sp_prefill_workspace_bytes(dl, H, D, sp.SP_BF16)), dtype=torch.uint8, device=device)
+        ms = timed(lambda: sp.sp_superpose_prefill(q, k, v, dl, D ** -0.5, out, None, ws))
+        byt, flop = 4.0 * T * H * D * 2, 4.0 * D * H * lay.allowed_pairs()
+        iters.append({"round": r, "prefix_len": int(lay.max_pre_len), "paths_per_prompt": int(lay.n_paths // n_prompts),
+                      "tokens": int(T), "prefill_ms": ms, "frac_hbm": gb(byt, ms) / hbm,
+                      "useful_tflops": flop / (ms * 1e-3) / 1e12, "arith_intensity": flop / byt})
+        # the k kept documents of every prompt (here: its first k remaining paths) join the prefix
+        kept = np.stack([np.arange(lay.prompt_path_off[b], lay.prompt_path_off[b] + k_keep) for b in range(n_prompts)])
+        lay = next_round_layout(lay, kept)
+        del q, k, v, out
+        torch.cuda.empty_cache()
+    print(json.dumps({"widened": True, "alibi": alibi,
+                      "iterative": {"prompts": n_prompts, "documents": n_docs, "kept_per_round": k_keep, "rounds": iters,
+                                    "data": "synthetic, lengths U{60..180}"}}))
+
+
+# ---------------------------------------------------------------------------------------
 def oracle_sample_pass(cfg, n_prompts):
     """Returns a closure that runs the whole hot path in the CPU oracle on the first n_prompts
     prompts of the workload, and the useful prefill FLOPs of that sample."""
@@ -646,13 +731,16 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch the decode loop eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling aid)")
+    ap.add_argument("--widened", action="store_true", help="time the ALiBi variants and an iterative-superposition workload instead of the step")
     ap.add_argument("--no-extra", action="store_true", help="skip the cfg3 / cfg4 passes that follow the default workload")
     ap.add_argument("--prompts", type=int, default=None, help="override the prompts per GPU (profiling aid)")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the decode steps (profiling aid)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         raise SystemExit(subprocess.call(launcher_command(args.gpus, sys.argv[1:])))
-    if args.impl == "reference":
+    if args.widened:
+        run_widened(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -354,6 +354,13 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     slope_l2 = p.slopes[c.h] * kLog2eT;
                 }
             }
+            // ALiBi: lane i fetches the positions of keys i and 32 + i of the tile (ahead of the wait,
+            // off the chain); the chunk loops read them with shuffles instead of 64 loads per thread
+            float kp0 = 0.f, kp1 = 0.f;
+            if (ALIBI) {
+                if (lane < kt.n_valid) kp0 = __ldg(p.pos + kt.row0 + lane);
+                if (32 + lane < kt.n_valid) kp1 = __ldg(p.pos + kt.row0 + 32 + lane);
+            }
             if (!(ok = mbar_wait_warp(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
             tc_fence_after();
 
@@ -368,10 +375,11 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 uint32_t r[kCh];
                 tmem_ldc(s_addr + ch * kCh, r);
                 tmem_ld_wait();
-                if (ALIBI) {            // score * scale - slope * |distance|, every thread reads the same key positions
+                if (ALIBI) {            // score * scale - slope * |distance|; key positions come from the lanes' registers
+                    const float kp = ch < 2 ? kp0 : kp1;
 #pragma unroll
                     for (int i = 0; i < kCh; ++i) {
-                        const float pk = ch * kCh + i < kt.n_valid ? __ldg(p.pos + kt.row0 + ch * kCh + i) : 0.f;
+                        const float pk = __shfl_sync(0xffffffffu, kp, (ch & 1) * kCh + i);
                         r[i] = __float_as_uint(fmaf(__uint_as_float(r[i]), sc, -slope_l2 * fabsf(pq - pk)));
                     }
                 }
@@ -421,9 +429,10 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                         tmem_ldc(s_addr + ch * kCh, r);
                         tmem_ld_wait();
                         if (ALIBI) {
+                            const float kp = ch < 2 ? kp0 : kp1;
 #pragma unroll
                             for (int i = 0; i < kCh; ++i) {
-                                const float pkey = ch * kCh + i < kt.n_valid ? __ldg(p.pos + kt.row0 + ch * kCh + i) : 0.f;
+                                const float pkey = __shfl_sync(0xffffffffu, kp, (ch & 1) * kCh + i);
                                 r[i] = __float_as_uint(fmaf(__uint_as_float(r[i]), sc, -slope_l2 * fabsf(pq - pkey)));
                             }
                         }
