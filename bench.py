@@ -639,7 +639,21 @@ def run_widened(args):
         lay = next_round_layout(lay, kept)
         del q, k, v, out
         torch.cuda.empty_cache()
-    print(json.dumps({"widened": True, "alibi": alibi,
+    # bf16 with head_dim 64 (served by the fp32-arithmetic SIMT kernel): a smaller batch of the cfg2 shape
+    lay64 = draw_lengths(get_config("cfg2"), n_prompts=8)
+    T64, H64, D64 = lay64.total_tokens, 32, 64
+    g = torch.Generator(device=device); g.manual_seed(64)
+    q, k, v = (torch.randn(T64, H64, D64, device=device, generator=g).mul_(D64 ** -0.5).bfloat16() for _ in range(3))
+    out = torch.empty_like(q)
+    dl64 = sp.DeviceLayout.from_host(lay64, device)
+    ws64 = torch.zeros(max(256, sp.sp_prefill_workspace_bytes(dl64, H64, D64, sp.SP_BF16)), dtype=torch.uint8, device=device)
+    ms64 = timed(lambda: sp.sp_superpose_prefill(q, k, v, dl64, D64 ** -0.5, out, None, ws64), reps=3)
+    flop64 = 4.0 * D64 * H64 * lay64.allowed_pairs()
+    simt = {"shape": "cfg2 lengths, 8 prompts, 32 heads x 64, bf16", "tokens": int(T64), "prefill_ms": ms64,
+            "useful_tflops": flop64 / (ms64 * 1e-3) / 1e12, "frac_hbm": gb(4.0 * T64 * H64 * D64 * 2, ms64) / hbm,
+            "note": "warp per (row, head), fp32 FMA arithmetic, no tensor cores"}
+    del q, k, v, out
+    print(json.dumps({"widened": True, "alibi": alibi, "bf16_head_dim_64": simt,
                       "iterative": {"prompts": n_prompts, "documents": n_docs, "kept_per_round": k_keep, "rounds": iters,
                                     "data": "synthetic, lengths U{60..180}"}}))
 
