@@ -15,9 +15,15 @@ struct TcTile {                       // one query tile (shared by all heads)
     int32_t pad0, pad1;
 };
 
+struct PairRec {                      // up to two consecutive query tiles of one segment
+    int32_t tile0;                    // index of the first one in the tile list
+    int32_t n;                        // 1 or 2
+};
+
 struct TcHeader {                     // start of the workspace
     uint32_t status;
     uint32_t n_tiles;
+    uint32_t n_pairs;
 };
 
 // ---- plan: ragged layout -> tile list ---------------------------------------------------
@@ -30,6 +36,7 @@ struct PlanArgs {
     int64_t max_tiles;                // capacity of the tile list
     TcHeader *hdr;
     TcTile *tiles;
+    PairRec *pairs = nullptr;         // optional: the tiles grouped two by two per segment
 };
 
 // What the host cannot check, the plan kernel does: a segment whose device-side numbers
@@ -39,9 +46,9 @@ struct PlanArgs {
 
 static __global__ void __launch_bounds__(1024) prefill_plan_kernel(const PlanArgs a)
 {
-    __shared__ int warp_tot[32];
-    __shared__ int running;
-    if (threadIdx.x == 0) running = 0;
+    __shared__ int warp_tot[32], warp_tot2[32];
+    __shared__ int running, running2;
+    if (threadIdx.x == 0) { running = 0; running2 = 0; }
     __syncthreads();
     const int n_seq = a.n_prompts + a.n_paths;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -80,17 +87,28 @@ static __global__ void __launch_bounds__(1024) prefill_plan_kernel(const PlanArg
         }
         if (bad) a.hdr->status = STATUS_BAD_LAYOUT;
         const int nt = (rows + a.tile_rows - 1) / a.tile_rows;
-        int incl = nt;
+        const int np = (nt + 1) / 2;
+        int incl = nt, incl2 = np;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
+            const int v2 = __shfl_up_sync(0xffffffffu, incl2, o);
+            if (lane >= o) { incl += v; incl2 += v2; }
         }
-        if (lane == 31) warp_tot[warp] = incl;
+        if (lane == 31) { warp_tot[warp] = incl; warp_tot2[warp] = incl2; }
         __syncthreads();
-        int before = running;
-        for (int w = 0; w < warp; ++w) before += warp_tot[w];
+        int before = running, before2 = running2;
+        for (int w = 0; w < warp; ++w) { before += warp_tot[w]; before2 += warp_tot2[w]; }
         int off = before + incl - nt;
+        if (a.pairs) {
+            const int off2 = before2 + incl2 - np;
+            for (int t = 0; t < np && off + 2 * t < a.max_tiles; ++t) {
+                PairRec pr;
+                pr.tile0 = off + 2 * t;
+                pr.n = (2 * t + 1 < nt && off + 2 * t + 1 < a.max_tiles) ? 2 : 1;
+                a.pairs[off2 + t] = pr;
+            }
+        }
         for (int t = 0; t < nt && off + t < a.max_tiles; ++t) {
             TcTile tl;
             tl.q_off = first + t * a.tile_rows;
@@ -101,10 +119,13 @@ static __global__ void __launch_bounds__(1024) prefill_plan_kernel(const PlanArg
             a.tiles[off + t] = tl;
         }
         __syncthreads();
-        if (threadIdx.x == 1023) running = before + incl;
+        if (threadIdx.x == 1023) { running = before + incl; running2 = before2 + incl2; }
         __syncthreads();
     }
-    if (threadIdx.x == 0) a.hdr->n_tiles = (uint32_t)min((int64_t)running, a.max_tiles);
+    if (threadIdx.x == 0) {
+        a.hdr->n_tiles = (uint32_t)min((int64_t)running, a.max_tiles);
+        a.hdr->n_pairs = (uint32_t)min((int64_t)running2, a.max_tiles);
+    }
 }
 
 static inline int64_t plan_max_tiles(int n_prompts, int n_paths, int max_pre_len, int max_path_len, int tile_rows)

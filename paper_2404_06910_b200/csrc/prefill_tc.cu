@@ -17,6 +17,8 @@
 // share an SM (256 TMEM columns each).  A small plan kernel turns the ragged layout into a
 // tile list.  Every mbarrier wait is bounded: on expiry the block records a timeout in the
 // workspace status word, unwinds, frees its TMEM and exits.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "prefill_plan.cuh"
 #include "tc_ptx.cuh"
@@ -141,9 +143,13 @@ struct Cursor {
 // first O = P V may overwrite it.
 // V_CLEAN[st]: on a tile whose key count is not a multiple of 16, the rows of the V stage between the
 // last key and the end of the last 16-key MMA step have been zeroed (see the cleaner role).
+// V_SEEN[st]: the cleaner has passed this fill of the V stage.  The producer waits for it before the next
+// fill: a thread that waits on every fill of a barrier must be one of the parties the next fill
+// depends on, or it could fall two fills behind, where a parity wait answers for the wrong fill.
 enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_V_FULL = BAR_K_FULL + 2, BAR_S_FULL = BAR_V_FULL + 2,
        BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2, BAR_L_READY = BAR_O_DONE + 2,
-       BAR_X_FREE = BAR_L_READY + 2, BAR_O_FREE = BAR_X_FREE + 2, BAR_V_CLEAN, BAR_DRAIN = BAR_V_CLEAN + 2, BAR_COUNT };
+       BAR_X_FREE = BAR_L_READY + 2, BAR_O_FREE = BAR_X_FREE + 2, BAR_V_CLEAN, BAR_V_SEEN = BAR_V_CLEAN + 2,
+       BAR_DRAIN = BAR_V_SEEN + 2, BAR_COUNT };
 
 template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
@@ -204,7 +210,8 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     mbar_expect_tx(&bars[BAR_K_FULL + st], (32u << ks) * (kHD * 2));
                     tma_load_3d(sK + st * kKVBytes, &p.mk[ks], 0, kt.row0, hk * 2, &bars[BAR_K_FULL + st]);
                     ++nk[st];
-                    if (!(ok = mbar_wait(&bars[BAR_O_DONE + st], ph ^ 1))) break;       // V stage free
+                    if (!(ok = mbar_wait(&bars[BAR_O_DONE + st], ph ^ 1))) break;       // V stage free ...
+                    if (!(ok = mbar_wait(&bars[BAR_V_SEEN + st], ph ^ 1))) break;       // ... and passed by the cleaner
                     mbar_expect_tx(&bars[BAR_V_FULL + st], (32u << ks) * (kHD * 2));
                     tma_load_3d(sV + st * kKVBytes, &p.mv[ks], 0, kt.row0, hk * 2, &bars[BAR_V_FULL + st]);
                     ++nv[st];
@@ -303,7 +310,10 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 // every tile's phase is waited for (not only the ragged ones), so that this warp can
                 // never be a whole barrier phase ahead of the loads
                 if (!(ok = mbar_wait_warp(&bars[BAR_V_FULL + st], (c.g >> 1) & 1))) break;
-                if ((n_valid & 15) == 0) continue;
+                if ((n_valid & 15) == 0) {
+                    if (lane == 0) mbar_arrive(&bars[BAR_V_SEEN + st]);
+                    continue;
+                }
                 const int n_mma = (n_valid + 15) & ~15;
                 const int half_bytes = (32 << kv_box_sel(n_valid)) * 128;      // one 64-column half of the box
                 unsigned char *vs = sV + st * kKVBytes;
@@ -315,7 +325,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 }
                 fence_proxy_async();                 // generic-proxy stores -> visible to the MMA's reads
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bars[BAR_V_CLEAN + st]);
+                if (lane == 0) { mbar_arrive(&bars[BAR_V_CLEAN + st]); mbar_arrive(&bars[BAR_V_SEEN + st]); }
                 ++n_ragged[st];
             }
         }
@@ -567,6 +577,25 @@ static int encode_rows_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, 
     return SP_OK;
 }
 
+// The same view for the other TMA-fed kernels of the library.
+int make_rows_tensor_map(CUtensorMap *m, const void *base, int64_t rows, int64_t cols, int box_rows)
+{
+    static EncodeTiledFn enc = nullptr;
+    if (!enc) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        SP_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+        SP_REQUIRE(fn != nullptr && qres == cudaDriverEntryPointSuccess, SP_ERR_CUDA,
+                   "cuTensorMapEncodeTiled is not available from this driver");
+        enc = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    return encode_rows_map(enc, m, base, rows, cols, box_rows);
+}
+bool prefill_stall_hook() { return g_stall_producer; }
+int launch_prefill_pair(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos,
+                        const float *slopes, int n_heads, int n_kv_heads, float scale, void *out, float *lse,
+                        void *ws, cudaStream_t st);
+
 static int64_t max_tiles(int n_prompts, int n_paths, int max_pre_len, int max_path_len)
 {
     return plan_max_tiles(n_prompts, n_paths, max_pre_len, max_path_len, kBM);
@@ -575,13 +604,22 @@ static int64_t max_tiles(int n_prompts, int n_paths, int max_pre_len, int max_pa
 size_t prefill_tc_workspace_bytes(int n_prompts, int n_paths, int max_pre_len, int max_path_len, int)
 {
     if (n_prompts < 0 || n_paths < 0 || max_pre_len < 0 || max_path_len < 0) return 256;
-    return 256 + round_up((size_t)max_tiles(n_prompts, n_paths, max_pre_len, max_path_len) * sizeof(TcTile), 256);
+    const size_t cap = (size_t)max_tiles(n_prompts, n_paths, max_pre_len, max_path_len);
+    return 256 + round_up(cap * sizeof(TcTile), 256) + round_up(cap * sizeof(PairRec), 256);
 }
 
 int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos,
                       const float *slopes, int n_heads, int n_kv_heads, float scale, int rows, void *out,
                       float *lse, void *ws, size_t, cudaStream_t st)
 {
+    {
+        // Experimental variant (two query tiles of a segment per block, shared K/V stages; prefill_pair.cu).
+        // Parity-green and slower than this kernel on every workload measured, so it is off unless
+        // SP_B200_PREFILL_PAIR=1 is set when the library is first used.
+        static const bool use_pair = [] { const char *e = std::getenv("SP_B200_PREFILL_PAIR"); return e && e[0] == '1'; }();
+        if (use_pair && rows == SP_ROWS_ALL)
+            return launch_prefill_pair(q, k, v, lay, pos, slopes, n_heads, n_kv_heads, scale, out, lse, ws, st);
+    }
     static EncodeTiledFn enc = nullptr;
     if (!enc) {
         void *fn = nullptr;

@@ -736,3 +736,20 @@ def test_decode_long_sequences_many_splits():
     lay = build_layout([64], [[2000, 1500, 3000]], [[32, 32, 32]])
     _decode_case(lay, 2, 2, 128, "bf16", 3, [[2, 0, 1]], 40, [37], 550)
     _decode_case(lay, 1, 1, 64, "f32", 2, [[1, 2]], 8, [8], 551)
+
+
+def test_prefill_pair_variant_in_child_process():
+    """The experimental two-tiles-per-block prefill (shared K/V stages) is chosen by an environment
+    variable when the library is first used, so it runs in a child process: the ragged, sub-tile,
+    peaky, random-layout, determinism and ALiBi prefill cases against the oracle."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, SP_B200_PREFILL_PAIR="1")
+    r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu", "-p", "no:cacheprovider",
+                        os.path.join(root, "tests", "test_gpu_parity.py"), os.path.join(root, "tests", "test_gpu_independence.py"),
+                        "-k", "(prefill and not query and not pair_variant) or paths_do_not or rows_outside"],
+                       env=env, capture_output=True, text=True, timeout=1200, cwd=root)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
+    assert " passed" in r.stdout
