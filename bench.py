@@ -639,6 +639,33 @@ def run_widened(args):
         lay = next_round_layout(lay, kept)
         del q, k, v, out
         torch.cuda.empty_cache()
+    # grouped query heads: the cfg2 decode shape with 8 KV heads under the 32 query heads (one block owns
+    # a KV head and 4 of its query heads, so each K / V row is read once per group)
+    lay_g = draw_lengths(cfg)
+    Bg, Hkv_g, n_g = lay_g.n_prompts, 8, 8
+    g = torch.Generator(device=device); g.manual_seed(8)
+    mk = lambda *shape: torch.randn(*shape, device=device, generator=g).mul_(D ** -0.5).bfloat16()
+    kc_sets = [(mk(lay_g.total_tokens, Hkv_g, D), mk(lay_g.total_tokens, Hkv_g, D)) for _ in range(4)]   # > 2 x L2 in rotation
+    qg, tkg, tvg = mk(n_g, Bg, H, D), mk(Bg, n_g, Hkv_g, D), mk(Bg, n_g, Hkv_g, D)
+    dl_g = sp.DeviceLayout.from_host(lay_g, device)
+    kept_g = torch.stack([torch.arange(2, dtype=torch.int32) + int(lay_g.prompt_path_off[b]) for b in range(Bg)]).to(device)
+    tl_g = torch.arange(1, n_g + 1, dtype=torch.int32)[:, None].expand(n_g, Bg).contiguous().to(device)
+    out_g = torch.empty((n_g, Bg, H, D), dtype=torch.bfloat16, device=device)
+    ws_g = torch.zeros(max(256, sp.sp_decode_workspace_bytes(Bg, H, D)), dtype=torch.uint8, device=device)
+    def dec_gqa():
+        for t in range(n_g):
+            kc, vc = kc_sets[t % len(kc_sets)]
+            sp.sp_pruned_decode(qg[t], kc, vc, dl_g, kept_g, 2, tkg, tvg, tl_g[t], n_g, D ** -0.5, out_g[t], None, ws_g)
+    gqa_ms = timed(dec_gqa, reps=5, per=n_g)
+    keys_g = sum(int(lay_g.pre_len[b]) + sum(int(lay_g.doc_len[i] + lay_g.qry_len[i]) for i in kept_g[b].tolist()) for b in range(Bg)) \
+        + Bg * (n_g + 1) / 2.0
+    bytes_g = keys_g * 2 * Hkv_g * D * 2
+    gqa = {"shape": "cfg2 lengths, 64 prompts, 32 query heads over 8 KV heads, k = 2", "decode_us": gqa_ms * 1e3,
+           "algorithmic_mb": bytes_g / 1e6, "frac_hbm": gb(bytes_g, gqa_ms) / hbm,
+           "note": "bytes counted once per KV head; launches issued eagerly, KV sets rotating"}
+    del kc_sets, qg, tkg, tvg, out_g
+    torch.cuda.empty_cache()
+
     # bf16 with head_dim 64 (served by the fp32-arithmetic SIMT kernel): a smaller batch of the cfg2 shape
     lay64 = draw_lengths(get_config("cfg2"), n_prompts=8)
     T64, H64, D64 = lay64.total_tokens, 32, 64
@@ -653,7 +680,7 @@ def run_widened(args):
             "useful_tflops": flop64 / (ms64 * 1e-3) / 1e12, "frac_hbm": gb(4.0 * T64 * H64 * D64 * 2, ms64) / hbm,
             "note": "warp per (row, head), fp32 FMA arithmetic, no tensor cores"}
     del q, k, v, out
-    print(json.dumps({"widened": True, "alibi": alibi, "bf16_head_dim_64": simt,
+    print(json.dumps({"widened": True, "alibi": alibi, "decode_grouped_heads": gqa, "bf16_head_dim_64": simt,
                       "iterative": {"prompts": n_prompts, "documents": n_docs, "kept_per_round": k_keep, "rounds": iters,
                                     "data": "synthetic, lengths U{60..180}"}}))
 
