@@ -11,9 +11,14 @@
 //   O += P V      tcgen05.mma with A = P from TMEM, B = V from shared memory (MN-major)
 // Roles (warpgroups of 4 warps, registers rebalanced with setmaxnreg): warps 0-3 softmax,
 // warps 4-7 epilogue (O / l -> bf16 -> global, LSE) off the softmax warps' critical path,
-// warp 8 TMA producer, warp 9 MMA issuer / TMEM owner, warps 10-11 idle.
-// K and V tiles are double-buffered in shared memory and S in TMEM, so the next S = Q K^T is
-// issued while the softmax of the current tile runs.  The grid is persistent; two blocks
+// warp 8 loads Q and K (TMA), warp 9 issues S = Q K^T and owns the TMEM allocation, warp 10 loads V
+// (TMA) and cleans ragged V tiles, warp 11 issues O += P V.  The two products have an issuing thread
+// each: one thread doing both was the busiest thread of the block (waits, work-list arithmetic and
+// MMA issue back-pressure of two products in series), and every delay of it went straight into the
+// softmax warps' wait for S.  The two threads' MMAs are ordered through mbarriers only where they
+// touch the same tensor memory (S of tile g+2 overwrites P of tile g).
+// K and V tiles are double-buffered in shared memory and S in TMEM, so the S = Q K^T of the next two
+// tiles is issued while the softmax of the current tile runs.  The grid is persistent; two blocks
 // share an SM (256 TMEM columns each).  A small plan kernel turns the ragged layout into a
 // tile list.  Every mbarrier wait is bounded: on expiry the block records a timeout in the
 // workspace status word, unwinds, frees its TMEM and exits.
@@ -30,8 +35,8 @@ using namespace ptx;
 constexpr int kBM = 128;              // query rows per tile
 constexpr int kBN = 64;               // keys per tile
 constexpr int kHD = 128;              // head_dim
-constexpr int kTmaWarp = 8, kMmaWarp = 9, kCleanWarp = 10;
-constexpr int kTcThreads = 12 * 32;   // warps 0-3 softmax, 4-7 epilogue, 8 producer, 9 MMA issuer, 10-11 idle (warpgroup padding)
+constexpr int kTmaWarp = 8, kMmaWarp = 9, kCleanWarp = 10, kPvWarp = 11;
+constexpr int kTcThreads = 12 * 32;   // warps 0-3 softmax, 4-7 epilogue, 8 Q/K loads, 9 S issuer, 10 V loads + cleaning, 11 P V issuer
 constexpr int kQBytes = kBM * kHD * 2;     // 32 KB
 constexpr int kKVBytes = kBN * kHD * 2;    // 16 KB per stage
 constexpr int kTmemCols = 256;        // S/P double buffer: [0,64) [64,128)   O: [128,256)
@@ -132,8 +137,9 @@ struct Cursor {
     __device__ __forceinline__ bool last_of_item() const { return j == n_kv - 1; }
 };
 
-// S_FULL[st] (S = Q K^T of a tile complete) also tells the producer that K stage st is free;
-// O_DONE[st] (O += P V complete) also frees V stage st: one tcgen05.commit serves both waiters.
+// S_FULL[st] (S = Q K^T of a tile complete) also tells the Q/K loader that K stage st is free;
+// O_DONE[st] (O += P V complete) also frees V stage st for the V loader and the S / P columns st for
+// the S issuer: one tcgen05.commit serves all waiters.
 // L_READY[item parity]: the softmax warps have published an item's row sums; X_FREE[item parity]:
 // the epilogue warps have read them, so the slot may be rewritten two items later.  Both are
 // per-parity pairs because warps whose rows are masked out of a tile finish it almost at once:
@@ -143,13 +149,15 @@ struct Cursor {
 // first O = P V may overwrite it.
 // V_CLEAN[st]: on a tile whose key count is not a multiple of 16, the rows of the V stage between the
 // last key and the end of the last 16-key MMA step have been zeroed (see the cleaner role).
-// V_SEEN[st]: the cleaner has passed this fill of the V stage.  The producer waits for it before the next
-// fill: a thread that waits on every fill of a barrier must be one of the parties the next fill
-// depends on, or it could fall two fills behind, where a parity wait answers for the wrong fill.
+// Every thread that waits on a double-buffered barrier waits on each of its fills in order and is one of
+// the parties the next fill depends on (the V loader is also the cleaner; the S issuer's wait for
+// O_DONE gates the S whose softmax gates the next O += P V): a waiter that skipped fills could be two
+// ahead, one that nothing waits for could fall two behind, and a parity wait would then answer for the
+// wrong fill.
 enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_V_FULL = BAR_K_FULL + 2, BAR_S_FULL = BAR_V_FULL + 2,
        BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2, BAR_L_READY = BAR_O_DONE + 2,
-       BAR_X_FREE = BAR_L_READY + 2, BAR_O_FREE = BAR_X_FREE + 2, BAR_V_CLEAN, BAR_V_SEEN = BAR_V_CLEAN + 2,
-       BAR_DRAIN = BAR_V_SEEN + 2, BAR_COUNT };
+       BAR_X_FREE = BAR_L_READY + 2, BAR_O_FREE = BAR_X_FREE + 2, BAR_V_CLEAN, BAR_DRAIN = BAR_V_CLEAN + 2,
+       BAR_COUNT = BAR_DRAIN + 2 };      // DRAIN: one per issuing thread
 
 template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
@@ -187,21 +195,15 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
     bool ok = true;
 
     if (warp >= 8) {
-        reg_dealloc<56>();              // warps 8-11: producer, MMA issuer and two idle warps
+        reg_dealloc<56>();              // warps 8-11: the two loaders and the two MMA issuers
         if (warp == kTmaWarp) {
-            // -------------------------------------------------------------- TMA producer
+            // -------------------------------------------------------------- Q and K loads (TMA)
             if (lane == 0) {
-                uint32_t nq = 0, nk[2] = {0, 0}, nv[2] = {0, 0};     // loads issued per "full" barrier
+                uint32_t nq = 0, nk[2] = {0, 0};     // loads issued per "full" barrier
                 Cursor c;
+#pragma unroll 1
                 for (c.init(p.tiles, n_items, p.n_heads); c.valid && ok && !p.stall_producer; c.next()) {
                     const int hk = c.h / p.kv_group;
-                    if (c.j == 0) {
-                        if (!(ok = mbar_wait(&bars[BAR_Q_EMPTY], (c.item_no & 1) ^ 1))) break;
-                        const int qs = q_box_sel(c.t.n_rows);
-                        mbar_expect_tx(&bars[BAR_Q_FULL], (32u << qs) * (kHD * 2));
-                        tma_load_3d(sQ, &p.mq[qs], 0, c.t.q_row, c.h * 2, &bars[BAR_Q_FULL]);
-                        ++nq;
-                    }
                     const KvTile kt = c.kv();
                     const int st = c.g & 1;
                     const uint32_t ph = (c.g >> 1) & 1;
@@ -210,110 +212,103 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     mbar_expect_tx(&bars[BAR_K_FULL + st], (32u << ks) * (kHD * 2));
                     tma_load_3d(sK + st * kKVBytes, &p.mk[ks], 0, kt.row0, hk * 2, &bars[BAR_K_FULL + st]);
                     ++nk[st];
-                    if (!(ok = mbar_wait(&bars[BAR_O_DONE + st], ph ^ 1))) break;       // V stage free ...
-                    if (!(ok = mbar_wait(&bars[BAR_V_SEEN + st], ph ^ 1))) break;       // ... and passed by the cleaner
-                    mbar_expect_tx(&bars[BAR_V_FULL + st], (32u << ks) * (kHD * 2));
-                    tma_load_3d(sV + st * kKVBytes, &p.mv[ks], 0, kt.row0, hk * 2, &bars[BAR_V_FULL + st]);
-                    ++nv[st];
+                    if (c.j == 0) {
+                        // the item's query tile, after its first K tile: the Q slot is the later of the two to come free
+                        if (!(ok = mbar_wait(&bars[BAR_Q_EMPTY], (c.item_no & 1) ^ 1))) break;
+                        const int qs = q_box_sel(c.t.n_rows);
+                        mbar_expect_tx(&bars[BAR_Q_FULL], (32u << qs) * (kHD * 2));
+                        tma_load_3d(sQ, &p.mq[qs], 0, c.t.q_row, c.h * 2, &bars[BAR_Q_FULL]);
+                        ++nq;
+                    }
                 }
                 if (!ok) {
                     // a wait ran out: before the block may exit, its own copies in flight must
                     // have landed (bounded waits on the phase of the last load of each buffer)
                     if (nq) mbar_wait(&bars[BAR_Q_FULL], (nq - 1) & 1);
-                    for (int st = 0; st < 2; ++st) {
+                    for (int st = 0; st < 2; ++st)
                         if (nk[st]) mbar_wait(&bars[BAR_K_FULL + st], (nk[st] - 1) & 1);
-                        if (nv[st]) mbar_wait(&bars[BAR_V_FULL + st], (nv[st] - 1) & 1);
-                    }
                 }
             }
         } else if (warp == kMmaWarp) {
-            // -------------------------------------------------------------- MMA issuer
+            // -------------------------------------------------------------- MMA issuer, S = Q K^T
             if (lane == 0) {
                 // Descriptor words are loop-invariant up to a small address offset: build them once.
                 // High word: stride-dimension offset 1024 B (8-row groups), descriptor version 1, 128B swizzle.
                 const uint32_t d_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
                 const uint32_t q_lo = ((smem_u32(sQ) & 0x3ffffu) >> 4) | (1u << 16);
                 const uint32_t k_lo = ((smem_u32(sK) & 0x3ffffu) >> 4) | (1u << 16);
-                const uint32_t v_lo = (smem_u32(sV) & 0x3ffffu) >> 4;     // leading-dimension offset (half stride) added per tile
-                const uint32_t id_o = idesc_bf16(kBM, kHD, 0, 1);
-                uint32_t n_ragged[2] = {0, 0};      // ragged tiles seen per V stage (phase of V_CLEAN)
-                Cursor cs, cp;                      // cs: next S = Q K^T to issue; cp: next O += P V to issue
-                cs.init(p.tiles, n_items, p.n_heads);
-                cp.init(p.tiles, n_items, p.n_heads);
-
-                while (cp.valid && ok) {
-                    // S = Q K^T: the current tile's must be issued; the next tile's is issued one
-                    // ahead of the softmax as soon as its operands have landed
-                    while (cs.valid && (cs.g == cp.g ||
-                                        (cs.g == cp.g + 1 && (cs.j != 0 || mbar_test(&bars[BAR_Q_FULL], cs.item_no & 1)) &&
-                                         mbar_test(&bars[BAR_K_FULL + (cs.g & 1)], (cs.g >> 1) & 1)))) {
-                        const uint32_t st = cs.g & 1;
-                        if (cs.j == 0 && !(ok = mbar_wait(&bars[BAR_Q_FULL], cs.item_no & 1))) break;
-                        if (!(ok = mbar_wait(&bars[BAR_K_FULL + st], (cs.g >> 1) & 1))) break;
-                        tc_fence_after();
-                        const int n_valid = cs.kv().n_valid;
-                        const int n_mma = (n_valid + 15) & ~15;
-                        const uint32_t id_s = idesc_bf16(kBM, 0, 0, 0) | ((uint32_t)(n_mma >> 3) << 17);
-                        const uint32_t kb = k_lo + st * (kKVBytes >> 4);
-                        const uint32_t d = tb + st * kBN;
-                        // second 64-column half of a box: box_rows x 128 bytes further on (in 16-byte units)
-                        const uint32_t q_half = (32u << q_box_sel(cs.t.n_rows)) * 8u;
-                        const uint32_t k_half = (32u << kv_box_sel(n_valid)) * 8u;
-#pragma unroll
-                        for (int kk = 0; kk < kHD / 16; ++kk)              // contraction over head_dim
-                            umma_ss_lh(d, q_lo + (kk >> 2) * q_half + (kk & 3) * 2,
-                                       kb + (kk >> 2) * k_half + (kk & 3) * 2, d_hi, id_s, kk > 0 ? 1u : 0u);
-                        umma_commit(&bars[BAR_S_FULL + st]);
-                        if (cs.last_of_item()) umma_commit(&bars[BAR_Q_EMPTY]);
-                        cs.next();
-                    }
-                    if (!ok) break;
-                    const uint32_t st = cp.g & 1;
-                    const uint32_t ph = (cp.g >> 1) & 1;
-                    const int pv_valid = cp.kv().n_valid;
-                    const int n_k = (pv_valid + 15) >> 4;                 // 16-key steps
-                    if (!(ok = mbar_wait(&bars[BAR_P_FULL + st], ph))) break;
-                    if (!(ok = mbar_wait(&bars[BAR_V_FULL + st], ph))) break;
-                    if ((pv_valid & 15) && !(ok = mbar_wait(&bars[BAR_V_CLEAN + st], n_ragged[st]++ & 1))) break;
-                    // the first O = P V of an item overwrites O: the previous item's must have been read out
-                    if (cp.j == 0 && cp.item_no > 0 && !(ok = mbar_wait(&bars[BAR_O_FREE], (cp.item_no - 1) & 1))) break;
+                Cursor cs;                          // next S = Q K^T to issue
+#pragma unroll 1
+                for (cs.init(p.tiles, n_items, p.n_heads); cs.valid && ok; cs.next()) {
+                    const uint32_t st = cs.g & 1;
+                    if (cs.j == 0 && !(ok = mbar_wait(&bars[BAR_Q_FULL], cs.item_no & 1))) break;
+                    if (!(ok = mbar_wait(&bars[BAR_K_FULL + st], (cs.g >> 1) & 1))) break;
+                    // S(g) lands on the columns of P(g-2): the O += P V that reads them (issued by the other
+                    // issuing thread) must be complete
+                    if (cs.g >= 2 && !(ok = mbar_wait(&bars[BAR_O_DONE + st], ((cs.g >> 1) - 1) & 1))) break;
                     tc_fence_after();
-                    const uint32_t vb = (v_lo + st * (kKVBytes >> 4)) | (((32u << kv_box_sel(pv_valid)) * 8u) << 16);
-                    const uint32_t pa = tb + st * kBN;
+                    const int n_valid = cs.kv().n_valid;
+                    const int n_mma = (n_valid + 15) & ~15;
+                    const uint32_t id_s = idesc_bf16(kBM, 0, 0, 0) | ((uint32_t)(n_mma >> 3) << 17);
+                    const uint32_t kb = k_lo + st * (kKVBytes >> 4);
+                    const uint32_t d = tb + st * kBN;
+                    // second 64-column half of a box: box_rows x 128 bytes further on (in 16-byte units)
+                    const uint32_t q_half = (32u << q_box_sel(cs.t.n_rows)) * 8u;
+                    const uint32_t k_half = (32u << kv_box_sel(n_valid)) * 8u;
 #pragma unroll
-                    for (int kk = 0; kk < kBN / 16; ++kk)                 // contraction over keys
-                        if (kk < n_k)
-                            umma_ts_lh(tb + 128, pa + kk * 8, vb + kk * (2048 >> 4), d_hi, id_o, (cp.j > 0 || kk > 0) ? 1u : 0u);
-                    umma_commit(&bars[BAR_O_DONE + st]);
-                    cp.next();
+                    for (int kk = 0; kk < kHD / 16; ++kk)              // contraction over head_dim
+                        umma_ss_lh(d, q_lo + (kk >> 2) * q_half + (kk & 3) * 2,
+                                   kb + (kk >> 2) * k_half + (kk & 3) * 2, d_hi, id_s, kk > 0 ? 1u : 0u);
+                    umma_commit(&bars[BAR_S_FULL + st]);
+                    if (cs.last_of_item()) umma_commit(&bars[BAR_Q_EMPTY]);
                 }
                 if (!ok) {
-                    // a wait ran out: let every MMA already issued finish (bounded) before the
+                    // a wait ran out: let every MMA this thread issued finish (bounded) before the
                     // tensor memory they write is freed
                     umma_commit(&bars[BAR_DRAIN]);
                     mbar_wait(&bars[BAR_DRAIN], 0);
                 }
             }
-        } else if (warp == kCleanWarp) {
-            // -------------------------------------------------------------- V cleaner
-            // O += P V contracts over the keys rounded up to 16.  The rows of the V stage past the
-            // tile's last key hold whatever follows in the packed tensor (another path's rows);
-            // their P is exactly zero, but 0 x Inf or 0 x NaN would still reach O.  This warp
-            // zeroes those rows before the issuer may use the stage, so a path's output depends on
-            // nothing outside its own keys (Section 3.2: paths do not see each other).
-            uint32_t n_ragged[2] = {0, 0};
-            Cursor c;
+        } else if (warp == kPvWarp) {
+            // -------------------------------------------------------------- MMA issuer, O += P V
+            if (lane == 0) {
+                const uint32_t d_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+                const uint32_t v_lo = (smem_u32(sV) & 0x3ffffu) >> 4;     // leading-dimension offset (half stride) added per tile
+                const uint32_t id_o = idesc_bf16(kBM, kHD, 0, 1);
+                uint32_t n_ragged[2] = {0, 0};      // ragged tiles seen per V stage (phase of V_CLEAN)
+                Cursor cp;
 #pragma unroll 1
-            for (c.init(p.tiles, n_items, p.n_heads); c.valid && ok; c.next()) {
-                const int n_valid = c.kv().n_valid;
-                const int st = c.g & 1;
-                // every tile's phase is waited for (not only the ragged ones), so that this warp can
-                // never be a whole barrier phase ahead of the loads
-                if (!(ok = mbar_wait_warp(&bars[BAR_V_FULL + st], (c.g >> 1) & 1))) break;
-                if ((n_valid & 15) == 0) {
-                    if (lane == 0) mbar_arrive(&bars[BAR_V_SEEN + st]);
-                    continue;
+                for (cp.init(p.tiles, n_items, p.n_heads); cp.valid && ok; cp.next()) {
+                    const uint32_t st = cp.g & 1;
+                    const uint32_t ph = (cp.g >> 1) & 1;
+                    const int pv_valid = cp.kv().n_valid;
+                    const int n_k = (pv_valid + 15) >> 4;                 // 16-key steps
+                    // everything but P first: P is what arrives last
+                    if (!(ok = mbar_wait(&bars[BAR_V_FULL + st], ph))) break;
+                    if ((pv_valid & 15) && !(ok = mbar_wait(&bars[BAR_V_CLEAN + st], n_ragged[st]++ & 1))) break;
+                    // the first O = P V of an item overwrites O: the previous item's must have been read out
+                    if (cp.j == 0 && cp.item_no > 0 && !(ok = mbar_wait(&bars[BAR_O_FREE], (cp.item_no - 1) & 1))) break;
+                    const uint32_t vb = (v_lo + st * (kKVBytes >> 4)) | (((32u << kv_box_sel(pv_valid)) * 8u) << 16);
+                    const uint32_t pa = tb + st * kBN;
+                    if (!(ok = mbar_wait(&bars[BAR_P_FULL + st], ph))) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < kBN / 16; ++kk)                 // contraction over keys
+                        if (kk < n_k)
+                            umma_ts_lh(tb + 128, pa + kk * 8, vb + kk * (2048 >> 4), d_hi, id_o, (cp.j > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(&bars[BAR_O_DONE + st]);
                 }
+                if (!ok) {
+                    umma_commit(&bars[BAR_DRAIN + 1]);
+                    mbar_wait(&bars[BAR_DRAIN + 1], 0);
+                }
+            }
+        } else if (warp == kCleanWarp) {
+            // -------------------------------------------------------------- V loader and cleaner
+            auto clean_tile = [&](uint32_t g, int n_valid) -> bool {
+                const int st = g & 1;
+                if (!mbar_wait_warp(&bars[BAR_V_FULL + st], (g >> 1) & 1)) return false;
+                if ((n_valid & 15) == 0) return true;
                 const int n_mma = (n_valid + 15) & ~15;
                 const int half_bytes = (32 << kv_box_sel(n_valid)) * 128;      // one 64-column half of the box
                 unsigned char *vs = sV + st * kKVBytes;
@@ -325,8 +320,47 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                 }
                 fence_proxy_async();                 // generic-proxy stores -> visible to the MMA's reads
                 __syncwarp();
-                if (lane == 0) { mbar_arrive(&bars[BAR_V_CLEAN + st]); mbar_arrive(&bars[BAR_V_SEEN + st]); }
-                ++n_ragged[st];
+                if (lane == 0) mbar_arrive(&bars[BAR_V_CLEAN + st]);
+                return true;
+            };
+            // O += P V contracts over the keys rounded up to 16.  The rows of the V stage past the
+            // tile's last key hold whatever follows in the packed tensor (another path's rows);
+            // their P is exactly zero, but 0 x Inf or 0 x NaN would still reach O.  This warp
+            // zeroes those rows before the issuer may use the stage, so a path's output depends on
+            // nothing outside its own keys (Section 3.2: paths do not see each other).
+            // The same warp loads V: tile t goes into its stage as soon as O += P V of tile t-2 (the
+            // stage's previous user) is complete, then tile t-1, loaded one turn earlier, is waited for and
+            // cleaned.  Loading and cleaning in one thread keeps every V barrier's waits in fill order.
+            Cursor c;
+            int prev_valid = 0;                   // keys of tile t-1; 0: no such tile
+            uint32_t t_issued = 0;
+            c.init(p.tiles, n_items, p.n_heads);
+#pragma unroll 1
+            while (ok && (c.valid || prev_valid)) {
+                if (c.valid) {
+                    const int st = c.g & 1;
+                    if (c.g >= 2 && !(ok = mbar_wait_warp(&bars[BAR_O_DONE + st], ((c.g >> 1) - 1) & 1))) break;
+                    const KvTile kt = c.kv();
+                    if (lane == 0) {
+                        const int ks = kv_box_sel(kt.n_valid);
+                        mbar_expect_tx(&bars[BAR_V_FULL + st], (32u << ks) * (kHD * 2));
+                        tma_load_3d(sV + st * kKVBytes, &p.mv[ks], 0, kt.row0, (c.h / p.kv_group) * 2, &bars[BAR_V_FULL + st]);
+                    }
+                    ++t_issued;
+                    const int nv = kt.n_valid;
+                    // tile t-1
+                    if (prev_valid) ok = clean_tile(c.g - 1, prev_valid);
+                    prev_valid = nv;
+                    c.next();
+                } else {
+                    ok = clean_tile(c.g - 1, prev_valid);
+                    prev_valid = 0;
+                }
+            }
+            if (!ok && t_issued) {
+                // a wait ran out: the V copies in flight must land before the block exits (bounded)
+                mbar_wait_warp(&bars[BAR_V_FULL + ((t_issued - 1) & 1)], ((t_issued - 1) >> 1) & 1);
+                if (t_issued >= 2) mbar_wait_warp(&bars[BAR_V_FULL + ((t_issued - 2) & 1)], ((t_issued - 2) >> 1) & 1);
             }
         }
         __syncwarp();
