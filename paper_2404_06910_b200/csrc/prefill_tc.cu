@@ -200,6 +200,9 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             // -------------------------------------------------------------- Q and K loads (TMA)
             if (lane == 0) {
                 uint32_t nq = 0, nk[2] = {0, 0};     // loads issued per "full" barrier
+                // a query tile is read once: its lines may leave L2 first, which leaves more room for the K / V
+                // rows that the other query tiles of the path read again
+                const uint64_t pol_first = l2_policy_evict_first();
                 Cursor c;
 #pragma unroll 1
                 for (c.init(p.tiles, n_items, p.n_heads); c.valid && ok && !p.stall_producer; c.next()) {
@@ -217,7 +220,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                         if (!(ok = mbar_wait(&bars[BAR_Q_EMPTY], (c.item_no & 1) ^ 1))) break;
                         const int qs = q_box_sel(c.t.n_rows);
                         mbar_expect_tx(&bars[BAR_Q_FULL], (32u << qs) * (kHD * 2));
-                        tma_load_3d(sQ, &p.mq[qs], 0, c.t.q_row, c.h * 2, &bars[BAR_Q_FULL]);
+                        tma_load_3d_hint(sQ, &p.mq[qs], 0, c.t.q_row, c.h * 2, &bars[BAR_Q_FULL], pol_first);
                         ++nq;
                     }
                 }
@@ -567,8 +570,8 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                     for (int i = 0; i < 4; ++i) {
                         const int rr = (lane >> 2) + 8 * i, piece = lane & 3;
                         const uint4 w = *reinterpret_cast<const uint4 *>(stage + rr * 64 + ((piece ^ ((rr >> 1) & 3)) << 4));
-                        if (quad * 32 + rr < t.n_rows)
-                            *reinterpret_cast<uint4 *>(dst + (int64_t)(quad * 32 + rr) * row_pitch + cc * 64 + piece * 16) = w;
+                        if (quad * 32 + rr < t.n_rows)            // streaming store: the output is not read again here
+                            __stcs(reinterpret_cast<uint4 *>(dst + (int64_t)(quad * 32 + rr) * row_pitch + cc * 64 + piece * 16), w);
                     }
                     __syncwarp();
                 }
