@@ -212,6 +212,26 @@ int sp_pruned_decode(const void *q, const void *k_cache, const void *v_cache,
                      void *stream);
 
 /*
+ * The prefill with the rotation of Q folded in (Section 3.2.2, footnote on RoPE: the sinusoid's
+ * argument is evaluated at the interpolated position).  q arrives UNROTATED and is not modified:
+ * every 128-row query tile is rotated in shared memory, at the positions pos[T], between its
+ * arrival and its first use, with the arithmetic of sp_rope_apply (rot_dim = head_dim), so the
+ * result equals sp_rope_apply(q) followed by sp_superpose_prefill(rows = SP_ROWS_ALL) and one
+ * read and one write of Q are saved.  k must already be rotated (sp_rope_apply): it is the cache
+ * the decode step reads.  pos: fp32 [T] (sp_positions per prompt); base, pairing as for
+ * sp_rope_apply.  bf16 with head_dim 128 only; anything else returns SP_ERR_UNSUPPORTED (rotate
+ * with sp_rope_apply and call sp_superpose_prefill).  Workspace: sp_prefill_rope_workspace_bytes
+ * (the tile list plus a (cos, sin) table of total_tokens x 64 pairs, 512 bytes per token); the
+ * status word and sp_check_status work as for sp_superpose_prefill.
+ */
+size_t sp_prefill_rope_workspace_bytes(int n_prompts, int n_paths, int max_pre_len, int max_path_len,
+                                       int64_t total_tokens, int n_heads, int head_dim, int dtype);
+int sp_superpose_prefill_rope(const void *q, const void *k, const void *v, const sp_layout *lay,
+                              const float *pos, double base, int pairing, int n_heads, int n_kv_heads,
+                              int head_dim, float scale, void *out, float *lse, void *ws, size_t ws_bytes,
+                              int dtype, void *stream);
+
+/*
  * ALiBi variants (Section 3.2.2: the equilibrium assignment yields real-valued positions, which
  * the ALiBi encoding takes as they are; Section 3.2.1: with ALiBi, position gaps turn into
  * attention penalties, which is what the equilibrium assignment avoids).  They compute what

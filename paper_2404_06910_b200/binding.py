@@ -31,6 +31,7 @@ EXPORTS = (
     "sp_decode_workspace_bytes", "sp_pruned_decode", "sp_check_status",
     "sp_pruned_decode_static_max_bytes", "sp_pruned_decode_static",
     "sp_superpose_prefill_alibi", "sp_pruned_decode_alibi", "sp_rope_apply_pair", "sp_pruned_decode_rope",
+    "sp_prefill_rope_workspace_bytes", "sp_superpose_prefill_rope",
 )
 
 
@@ -73,6 +74,10 @@ def _load() -> ctypes.CDLL:
     lib.sp_prefill_workspace_bytes.argtypes = [c_int] * 7
     lib.sp_prefill_workspace_bytes.restype = sz
     lib.sp_superpose_prefill.argtypes = [vp, vp, vp, lp, c_int, c_int, c_int, c_f, c_int, vp, vp, vp, sz, c_int, vp]
+    lib.sp_prefill_rope_workspace_bytes.argtypes = [c_int, c_int, c_int, c_int, c_i64, c_int, c_int, c_int]
+    lib.sp_prefill_rope_workspace_bytes.restype = sz
+    lib.sp_superpose_prefill_rope.argtypes = [vp, vp, vp, lp, vp, c_d, c_int, c_int, c_int, c_int, c_f, vp, vp, vp, sz,
+                                              c_int, vp]
     lib.sp_path_scores_workspace_bytes.argtypes = [c_i64]
     lib.sp_path_scores_workspace_bytes.restype = sz
     lib.sp_path_scores.argtypes = [vp, c_i64, vp, vp, c_i64, c_int, c_int, vp, vp, vp, vp, vp, sz, c_int, vp]
@@ -215,6 +220,21 @@ def sp_superpose_prefill_alibi(q, k, v, lay: DeviceLayout, pos, slopes, scale: f
     _check(lib.sp_superpose_prefill_alibi(_ptr(q), _ptr(k), _ptr(v), ctypes.byref(lay.c), _ptr(pos), _ptr(slopes), H,
                                           Hkv, D, scale, rows, _ptr(out), _ptr(lse), _ptr(ws), _nbytes(ws),
                                           dtype_code(q), _stream(stream)))
+
+
+def sp_prefill_rope_workspace_bytes(lay: DeviceLayout, n_heads: int, head_dim: int, dtype: int) -> int:
+    return int(lib.sp_prefill_rope_workspace_bytes(lay.n_prompts, lay.n_paths, lay.max_pre_len, lay.max_path_len,
+                                                   lay.total_tokens, n_heads, head_dim, dtype))
+
+
+def sp_superpose_prefill_rope(q, k, v, lay: DeviceLayout, pos, base: float, pairing: int, scale: float, out, lse=None,
+                              ws=None, stream=None):
+    """sp_superpose_prefill over all rows with the rotation of the (unrotated) q folded in; k already rotated."""
+    T, H, D = q.shape
+    Hkv = k.shape[1]
+    _check(lib.sp_superpose_prefill_rope(_ptr(q), _ptr(k), _ptr(v), ctypes.byref(lay.c), _ptr(pos), base, pairing, H,
+                                         Hkv, D, scale, _ptr(out), _ptr(lse), _ptr(ws), _nbytes(ws), dtype_code(q),
+                                         _stream(stream)))
 
 
 def sp_path_scores_workspace_bytes(n_rows: int) -> int:

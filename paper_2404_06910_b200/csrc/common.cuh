@@ -41,7 +41,18 @@ int check_layout(const sp_layout *lay);     // host-visible fields only (api.cu)
 // Device status word codes (first 4 bytes of a workspace).
 enum : uint32_t { STATUS_OK = 0, STATUS_TIMEOUT = 1, STATUS_BAD_LAYOUT = 2 };
 
-int num_sms();                              // multiprocessors of the current device (api.cu)
+#ifdef __CUDACC__
+// One rotation (a, b) -> (a cos - b sin, a sin + b cos) with its roundings spelled out, so that every kernel that
+// rotates the same pair with the same (cos, sin) stores the same bits.
+__device__ __forceinline__ void rope_rotate(float a, float b, float c, float s, float &na, float &nb)
+{
+    na = __fmaf_rn(a, c, -__fmul_rn(b, s));
+    nb = __fmaf_rn(a, s, __fmul_rn(b, c));
+}
+#endif
+int num_sms();
+// (cos, sin) of every (token, pair m < rot_dim / 2) at pos * base^(-2m / rot_dim), [n_tokens][rot_dim / 2] (rope.cu).
+int launch_rope_table(const float *pos, int64_t n_tokens, int rot_dim, double base, float2 *out, cudaStream_t st);                              // multiprocessors of the current device (api.cu)
 
 // ---- device helpers ----------------------------------------------------------------
 #ifdef __CUDACC__

@@ -102,6 +102,8 @@ struct TcParams {
     int64_t total_tokens;
     float scale_log2e;
     const float *pos, *slopes;        // ALiBi variant: token positions [T], head slopes [H]
+    const float2 *rope_cs;            // ROPE variant: (cos, sin) of every (token, pair), [T][64]
+    int rope_pairing;
     int stall_producer;               // test hook: the producer issues no load, so every wait runs out
 };
 
@@ -185,7 +187,7 @@ struct Cursor {
 // wrong fill.
 enum { BAR_Q_FULL = 0, BAR_Q_EMPTY, BAR_K_FULL, BAR_V_FULL = BAR_K_FULL + 2, BAR_S_FULL = BAR_V_FULL + 2,
        BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2, BAR_L_READY = BAR_O_DONE + 2,
-       BAR_X_FREE = BAR_L_READY + 2, BAR_O_FREE = BAR_X_FREE + 2, BAR_V_CLEAN, BAR_DRAIN = BAR_V_CLEAN + 2,
+       BAR_X_FREE = BAR_L_READY + 2, BAR_O_FREE = BAR_X_FREE + 2, BAR_V_CLEAN, BAR_Q_ROT = BAR_V_CLEAN + 2, BAR_DRAIN,
        BAR_COUNT = BAR_DRAIN + 2 };      // DRAIN: one per issuing thread
 
 template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
@@ -193,7 +195,9 @@ template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("s
 
 // ALIBI: scores get -slope_h * |pos_q - pos_k| before the softmax (Section 3.2.2: real-valued
 // positions are no obstacle for ALiBi); the plain instantiation carries none of that code.
-template <bool ALIBI>
+// ROPE: Q arrives unrotated; the softmax warps rotate each query tile in shared memory, at the tokens' real-valued
+// positions (Section 3.2.2, footnote on RoPE), between its arrival and the item's first S = Q K^T.
+template <bool ALIBI, bool ROPE>
 __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_constant__ TcParams p)
 {
     extern __shared__ unsigned char smem_raw[];
@@ -210,7 +214,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int i = 0; i < BAR_COUNT; ++i)
-            mbar_init(&bars[i], ((i >= BAR_P_FULL && i < BAR_P_FULL + 2) || (i >= BAR_L_READY && i <= BAR_O_FREE)) ? 128 : 1);
+            mbar_init(&bars[i], ((i >= BAR_P_FULL && i < BAR_P_FULL + 2) || (i >= BAR_L_READY && i <= BAR_O_FREE) || i == BAR_Q_ROT) ? 128 : 1);
         fence_mbar_init();
         for (int i = 0; i < 3; ++i) prefetch_tmap(&p.mq[i]);
         for (int i = 0; i < 2; ++i) { prefetch_tmap(&p.mk[i]); prefetch_tmap(&p.mv[i]); }
@@ -273,7 +277,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
 #pragma unroll 1
                 for (cs.init(p.tiles, n_items, p.n_heads); cs.valid && ok; cs.next()) {
                     const uint32_t st = cs.g & 1;
-                    if (cs.j == 0 && !(ok = mbar_wait(&bars[BAR_Q_FULL], cs.item_no & 1))) break;
+                    if (cs.j == 0 && !(ok = mbar_wait(&bars[ROPE ? BAR_Q_ROT : BAR_Q_FULL], cs.item_no & 1))) break;
                     if (!(ok = mbar_wait(&bars[BAR_K_FULL + st], (cs.g >> 1) & 1))) break;
                     // S(g) lands on the columns of P(g-2): the O += P V that reads them (issued by the other
                     // issuing thread) must be complete
@@ -436,6 +440,55 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
             if (ALIBI) {
                 if (lane < kt.n_valid) kp0 = __ldg(p.pos + kt.row0 + lane);
                 if (32 + lane < kt.n_valid) kp1 = __ldg(p.pos + kt.row0 + 32 + lane);
+            }
+            if (ROPE && first) {
+                // This thread's row of the new query tile: 8 pieces of 16 bytes in each 64-column half (the 128-byte
+                // swizzle permutes the pieces of a row by its index mod 8); the (cos, sin) pairs come from the
+                // per-token table.  The arithmetic is the standalone rotation's, so the tile equals what that
+                // kernel would have stored.
+                if (!(ok = mbar_wait_warp(&bars[BAR_Q_FULL], c.item_no & 1))) break;
+                if (row < t.n_rows) {
+                    unsigned char *h0 = sQ + row * 128, *h1 = h0 + (32 << q_box_sel(t.n_rows)) * 128;
+                    const float4 *tab = reinterpret_cast<const float4 *>(p.rope_cs + (int64_t)(t.q_row + row) * (kHD / 2));
+                    const bool half_split = p.rope_pairing == SP_ROPE_HALF_SPLIT;
+#pragma unroll 1
+                    for (int pc = 0; pc < 8; ++pc) {
+                        uint4 *pa = reinterpret_cast<uint4 *>(h0 + ((pc ^ (row & 7)) << 4));
+                        uint4 *pb = reinterpret_cast<uint4 *>(h1 + ((pc ^ (row & 7)) << 4));
+                        uint4 va = *pa, vb = *pb;
+                        uint32_t *ua = reinterpret_cast<uint32_t *>(&va), *ub = reinterpret_cast<uint32_t *>(&vb);
+                        if (half_split) {            // element j of the piece in half 0 pairs with element j in half 1
+#pragma unroll
+                            for (int j2 = 0; j2 < 4; ++j2) {
+                                const float4 w = __ldg(tab + pc * 4 + j2);      // pairs 8 pc + 2 j2, + 1
+                                const float a0 = __uint_as_float(ua[j2] << 16), a1 = __uint_as_float(ua[j2] & 0xffff0000u);
+                                const float b0 = __uint_as_float(ub[j2] << 16), b1 = __uint_as_float(ub[j2] & 0xffff0000u);
+                                float na0, nb0, na1, nb1;
+                                rope_rotate(a0, b0, w.x, w.y, na0, nb0);
+                                rope_rotate(a1, b1, w.z, w.w, na1, nb1);
+                                ua[j2] = pack_bf16x2(na0, na1);
+                                ub[j2] = pack_bf16x2(nb0, nb1);
+                            }
+                        } else {                     // neighbours pair up: pair 4 pc + j2 in half 0, 32 + 4 pc + j2 in half 1
+#pragma unroll
+                            for (int j2 = 0; j2 < 4; j2 += 2) {
+                                const float4 wa = __ldg(tab + pc * 2 + (j2 >> 1)), wb = __ldg(tab + 16 + pc * 2 + (j2 >> 1));
+                                float n0, n1;
+                                rope_rotate(__uint_as_float(ua[j2] << 16), __uint_as_float(ua[j2] & 0xffff0000u), wa.x, wa.y, n0, n1);
+                                ua[j2] = pack_bf16x2(n0, n1);
+                                rope_rotate(__uint_as_float(ua[j2 + 1] << 16), __uint_as_float(ua[j2 + 1] & 0xffff0000u), wa.z, wa.w, n0, n1);
+                                ua[j2 + 1] = pack_bf16x2(n0, n1);
+                                rope_rotate(__uint_as_float(ub[j2] << 16), __uint_as_float(ub[j2] & 0xffff0000u), wb.x, wb.y, n0, n1);
+                                ub[j2] = pack_bf16x2(n0, n1);
+                                rope_rotate(__uint_as_float(ub[j2 + 1] << 16), __uint_as_float(ub[j2 + 1] & 0xffff0000u), wb.z, wb.w, n0, n1);
+                                ub[j2 + 1] = pack_bf16x2(n0, n1);
+                            }
+                        }
+                        *pa = va; *pb = vb;
+                    }
+                }
+                fence_proxy_async();                 // generic-proxy stores -> visible to the MMA's reads
+                mbar_arrive(&bars[BAR_Q_ROT]);
             }
             if (!(ok = mbar_wait_warp(&bars[BAR_S_FULL + st], (c.g >> 1) & 1))) break;
             tc_fence_after();
@@ -680,16 +733,44 @@ size_t prefill_tc_workspace_bytes(int n_prompts, int n_paths, int max_pre_len, i
     return 256 + round_up(cap * sizeof(TcTile), 256) + round_up(cap * sizeof(PairRec), 256);
 }
 
+static int launch_tc(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos,
+                     const float *slopes, const float2 *rope_cs, int rope_pairing, int n_heads, int n_kv_heads,
+                     float scale, int rows, void *out, float *lse, void *ws, cudaStream_t st);
+
 int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos,
                       const float *slopes, int n_heads, int n_kv_heads, float scale, int rows, void *out,
                       float *lse, void *ws, size_t, cudaStream_t st)
+{
+    return launch_tc(q, k, v, lay, pos, slopes, nullptr, 0, n_heads, n_kv_heads, scale, rows, out, lse, ws, st);
+}
+
+// The (cos, sin) table of the ROPE variant sits behind the tile list and the pair list.
+size_t prefill_tc_rope_workspace_bytes(int n_prompts, int n_paths, int max_pre_len, int max_path_len, int64_t total_tokens)
+{
+    return prefill_tc_workspace_bytes(n_prompts, n_paths, max_pre_len, max_path_len, 0) +
+           round_up((size_t)std::max<int64_t>(total_tokens, 0) * (kHD / 2) * sizeof(float2), 256);
+}
+
+int launch_prefill_tc_rope(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos, double base,
+                           int pairing, int n_heads, int n_kv_heads, float scale, void *out, float *lse, void *ws,
+                           cudaStream_t st)
+{
+    float2 *table = reinterpret_cast<float2 *>(static_cast<char *>(ws) + prefill_tc_workspace_bytes(
+                        lay->n_prompts, lay->n_paths, lay->max_pre_len, lay->max_path_len, 0));
+    if (int rc = launch_rope_table(pos, lay->total_tokens, kHD, base, table, st)) return rc;
+    return launch_tc(q, k, v, lay, nullptr, nullptr, table, pairing, n_heads, n_kv_heads, scale, SP_ROWS_ALL, out, lse, ws, st);
+}
+
+static int launch_tc(const void *q, const void *k, const void *v, const sp_layout *lay, const float *pos,
+                     const float *slopes, const float2 *rope_cs, int rope_pairing, int n_heads, int n_kv_heads,
+                     float scale, int rows, void *out, float *lse, void *ws, cudaStream_t st)
 {
     {
         // Experimental variant (two query tiles of a segment per block, shared K/V stages; prefill_pair.cu).
         // Parity-green and slower than this kernel on every workload measured, so it is off unless
         // SP_B200_PREFILL_PAIR=1 is set when the library is first used.
         static const bool use_pair = [] { const char *e = std::getenv("SP_B200_PREFILL_PAIR"); return e && e[0] == '1'; }();
-        if (use_pair && rows == SP_ROWS_ALL)
+        if (use_pair && rows == SP_ROWS_ALL && !rope_cs)
             return launch_prefill_pair(q, k, v, lay, pos, slopes, n_heads, n_kv_heads, scale, out, lse, ws, st);
     }
     static EncodeTiledFn enc = nullptr;
@@ -730,18 +811,22 @@ int launch_prefill_tc(const void *q, const void *k, const void *v, const sp_layo
     p.n_heads = n_heads; p.kv_group = n_heads / n_kv_heads;
     p.total_tokens = lay->total_tokens; p.scale_log2e = scale * kLog2eT;
     p.pos = pos; p.slopes = slopes;
+    p.rope_cs = rope_cs; p.rope_pairing = rope_pairing;
     p.stall_producer = g_stall_producer ? 1 : 0;      // test hook, see sp_test_stall_producer below
 
     const int64_t items = max_tiles(lay->n_prompts, lay->n_paths, lay->max_pre_len, lay->max_path_len) * n_heads;
     if (items == 0) return SP_OK;
     const int grid = (int)std::min<int64_t>(items, 2 * num_sms());
     const int smem = kQBytes + 4 * kKVBytes + 4 * 2048 + 1024;
-    if (pos) {
-        SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        prefill_tc_kernel<true><<<grid, kTcThreads, smem, st>>>(p);
+    if (rope_cs) {
+        SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        prefill_tc_kernel<false, true><<<grid, kTcThreads, smem, st>>>(p);
+    } else if (pos) {
+        SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        prefill_tc_kernel<true, false><<<grid, kTcThreads, smem, st>>>(p);
     } else {
-        SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        prefill_tc_kernel<false><<<grid, kTcThreads, smem, st>>>(p);
+        SP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        prefill_tc_kernel<false, false><<<grid, kTcThreads, smem, st>>>(p);
     }
     SP_CUDA(cudaGetLastError());
     return SP_OK;

@@ -58,9 +58,7 @@ __device__ __forceinline__ void rotate_tokens(T *__restrict__ x, const float2 (*
 #pragma unroll
                 for (int j = 0; j < N; ++j) {
                     const float2 w = cs[t][m0 + j];
-                    const float na = a[j] * w.x - b[j] * w.y;
-                    const float nb = a[j] * w.y + b[j] * w.x;
-                    a[j] = na; b[j] = nb;
+                    rope_rotate(a[j], b[j], w.x, w.y, a[j], b[j]);
                 }
                 Pack<T>::store(pa, a);
                 Pack<T>::store(pb, b);
@@ -78,9 +76,7 @@ __device__ __forceinline__ void rotate_tokens(T *__restrict__ x, const float2 (*
 #pragma unroll
                 for (int j = 0; j < N; j += 2) {
                     const float2 w = cs[t][(e0 + j) >> 1];
-                    const float na = f[j] * w.x - f[j + 1] * w.y;
-                    const float nb = f[j] * w.y + f[j + 1] * w.x;
-                    f[j] = na; f[j + 1] = nb;
+                    rope_rotate(f[j], f[j + 1], w.x, w.y, f[j], f[j + 1]);
                 }
                 Pack<T>::store(p, f);
             }
@@ -96,8 +92,10 @@ __device__ __forceinline__ void rotate_tokens(T *__restrict__ x, const float2 (*
             T *pb = base + (pairing == SP_ROPE_HALF_SPLIT ? m + half : 2 * m + 1);
             const float a = to_float(*pa), b = to_float(*pb);
             const float2 w = cs[t][m];
-            store_val(pa, a * w.x - b * w.y);
-            store_val(pb, a * w.y + b * w.x);
+            float na, nb;
+            rope_rotate(a, b, w.x, w.y, na, nb);
+            store_val(pa, na);
+            store_val(pb, nb);
         }
     }
 }
@@ -187,6 +185,33 @@ static int rope_entry(const char *name, void *x, int64_t ld_token, int n_heads, 
     return dtype == SP_F32
                ? launch_rope<float>(x, x1, pos, n_tokens, ld_token, ld_token1, n_heads, n_heads1, head_dim, rot_dim, pairing, fr, st)
                : launch_rope<__nv_bfloat16>(x, x1, pos, n_tokens, ld_token, ld_token1, n_heads, n_heads1, head_dim, rot_dim, pairing, fr, st);
+}
+
+// The (cos, sin) of every (token, pair) as a table in device memory, for kernels that rotate tiles on the fly:
+// the same fp64 evaluation as above, so a tile rotated from the table equals one rotated by rope_kernel.
+__global__ void __launch_bounds__(256) rope_table_kernel(const float *__restrict__ pos, int64_t n_tokens, int half,
+                                                          float2 *__restrict__ out, const __grid_constant__ RopeFreq fr)
+{
+    const int64_t n = n_tokens * half;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t t = i / half;
+        const int m = (int)(i - t * half);
+        double s, c;
+        sincos((double)pos[t] * fr.inv_freq[m], &s, &c);
+        out[i] = make_float2((float)c, (float)s);
+    }
+}
+
+int launch_rope_table(const float *pos, int64_t n_tokens, int rot_dim, double base, float2 *out, cudaStream_t st)
+{
+    if (n_tokens <= 0) return SP_OK;
+    RopeFreq fr;
+    for (int m = 0; m < rot_dim / 2; ++m) fr.inv_freq[m] = std::pow(base, -2.0 * m / rot_dim);
+    const int64_t n = n_tokens * (rot_dim / 2);
+    const int grid = (int)std::min<int64_t>((n + 255) / 256, (int64_t)num_sms() * 16);
+    rope_table_kernel<<<grid, 256, 0, st>>>(pos, n_tokens, rot_dim / 2, out, fr);
+    SP_CUDA(cudaGetLastError());
+    return SP_OK;
 }
 
 }  // namespace sp
