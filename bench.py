@@ -594,6 +594,16 @@ def run_widened(args):
     plain_ms = timed(lambda: sp.sp_superpose_prefill(hp.q, hp.k, hp.v, hp.dl, hp.scale, hp.out, None, hp.ws_pre))
     alibi_ms = timed(lambda: sp.sp_superpose_prefill_alibi(hp.q, hp.k, hp.v, hp.dl, hp.pos, slopes, hp.scale, hp.out,
                                                            None, hp.ws_pre))
+    # the rotation of Q folded into the prefill (sp_superpose_prefill_rope) against the two calls it replaces
+    ws_rope = torch.zeros(sp.sp_prefill_rope_workspace_bytes(hp.dl, H, D, sp.SP_BF16), dtype=torch.uint8, device=device)
+    rope_q_ms = timed(lambda: sp.sp_rope_apply(hp.q, hp.pos, H, D, base=cfg.rope_base))
+    fused_ms = timed(lambda: sp.sp_superpose_prefill_rope(hp.q, hp.k, hp.v, hp.dl, hp.pos, cfg.rope_base,
+                                                          sp.SP_ROPE_HALF_SPLIT, hp.scale, hp.out, None, ws_rope))
+    rope_fused = {"workload": cfg.name, "rope_q_ms": rope_q_ms, "prefill_ms": plain_ms, "two_calls_ms": rope_q_ms + plain_ms,
+                  "prefill_rope_ms": fused_ms,
+                  "note": "sp_superpose_prefill_rope = (cos, sin) table kernel + tile plan + prefill kernel that rotates each "
+                          "query tile in shared memory; K is rotated by sp_rope_apply in both paths"}
+    del ws_rope
     hp.step()
     torch.cuda.synchronize()
     hp.bytes_decode = hp.decode_bytes()
@@ -680,7 +690,8 @@ def run_widened(args):
             "useful_tflops": flop64 / (ms64 * 1e-3) / 1e12, "frac_hbm": gb(4.0 * T64 * H64 * D64 * 2, ms64) / hbm,
             "note": "warp per (row, head), fp32 FMA arithmetic, no tensor cores"}
     del q, k, v, out
-    print(json.dumps({"widened": True, "alibi": alibi, "decode_grouped_heads": gqa, "bf16_head_dim_64": simt,
+    print(json.dumps({"widened": True, "alibi": alibi, "rope_folded_into_prefill": rope_fused, "decode_grouped_heads": gqa,
+                      "bf16_head_dim_64": simt,
                       "iterative": {"prompts": n_prompts, "documents": n_docs, "kept_per_round": k_keep, "rounds": iters,
                                     "data": "synthetic, lengths U{60..180}"}}))
 

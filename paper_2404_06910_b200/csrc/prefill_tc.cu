@@ -22,6 +22,8 @@
 // share an SM (256 TMEM columns each).  A small plan kernel turns the ragged layout into a
 // tile list.  Every mbarrier wait is bounded: on expiry the block records a timeout in the
 // workspace status word, unwinds, frees its TMEM and exits.
+// Compile-time variants: ALIBI adds the position bias to the scores; ROPE takes an unrotated Q and has the
+// softmax warps rotate each query tile in shared memory before its first use (sp_superpose_prefill_rope).
 #include <cstdlib>
 
 #include "common.cuh"
