@@ -513,6 +513,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                         const float pk = __shfl_sync(0xffffffffu, kp, (ch & 1) * kCh + i);
                         r[i] = __float_as_uint(fmaf(__uint_as_float(r[i]), sc, -slope_l2 * fabsf(pq - pk)));
                     }
+                    tmem_st16(s_addr + ch * kCh, r);     // the biased scores replace the raw ones: pass 2 reads them as they are
                 }
                 // keys past the row's limit (causal diagonal, ragged tail) -> -inf; skipped when the
                 // whole warp sees the whole chunk
@@ -523,6 +524,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
 #pragma unroll
                 for (int i = 0; i < kCh; i += 2) mx[(i >> 1) & 3] = fmax3(mx[(i >> 1) & 3], __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
             }
+            if (ALIBI) tmem_st_wait();                  // the biased scores are in place before pass 2 reads them
             const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc_exp;
             float alpha = 1.f;
             bool grow = false;
@@ -560,14 +562,6 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
                         uint32_t r[kCh];
                         tmem_ldc(s_addr + ch * kCh, r);
                         tmem_ld_wait();
-                        if (ALIBI) {
-                            const float kp = ch < 2 ? kp0 : kp1;
-#pragma unroll
-                            for (int i = 0; i < kCh; ++i) {
-                                const float pkey = __shfl_sync(0xffffffffu, kp, (ch & 1) * kCh + i);
-                                r[i] = __float_as_uint(fmaf(__uint_as_float(r[i]), sc, -slope_l2 * fabsf(pq - pkey)));
-                            }
-                        }
                         if (ch * kCh + 16 > lim0) {
 #pragma unroll
                             for (int i = 0; i < kCh; ++i) r[i] = (ch * kCh + i < lim) ? r[i] : 0xff800000u;
